@@ -1,0 +1,209 @@
+/* fdc.h - C ABI of the dependency-masked multi-branch decode path (B200, sm_100a).
+ *
+ * The method (FastDriveCoT): a chain-of-thought template is a DAG of fields; every field
+ * whose prerequisites are complete decodes one token in the same forward pass
+ * (Algorithm 1, Sec. 3.2).  All parallel fields are packed into ONE sequence sharing one KV
+ * cache; an attention mask derived from the graph lets a token attend a field iff that
+ * field is an ancestor of its own (Eq. 1, Sec. 3.3), fixed-length slots make every position
+ * id known in advance, and padding is visible to nobody and never processed (Sec. 3.3).
+ *
+ * One forward pass through this library, everything stream-ordered on the device:
+ *     fdc_frontier      Algorithm 1 body: retire finished fields, admit newly ready ones,
+ *                       emit this pass's packed branch list (node, token, KV row, position)
+ *     fdc_build_masks   Eq. 1 as per-branch row bitmaps + the list of KV tiles anyone sees
+ *     per layer:
+ *       fdc_kv_append   write each branch's new K/V vector at its slot row
+ *       fdc_decode_attn masked attention of all branches x all GQA heads of a scene over the
+ *                       shared cache, reading each visible KV row once (Sec. 3.3, "Reduced
+ *                       Memory Bottleneck"), split over the GPU and combined
+ *
+ * Conventions
+ *   - Every function returns FDC_OK (0) or a negative FDC_ERR_*; nothing throws, aborts or
+ *     traps.  Host-side argument errors are reported before anything is launched.
+ *   - "host" pointers are dereferenced by the calling thread; "device" pointers are only
+ *     handed to kernels.  All device buffers are CALLER-OWNED (sizes from fdc_plan_query /
+ *     fdc_attn_workspace_bytes); the library owns only the opaque fdc_plan.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = default stream).  fdc_state_init,
+ *     fdc_frontier, fdc_build_masks, fdc_kv_append and fdc_decode_attn only enqueue work;
+ *     they never synchronise or read device memory on the host.
+ *   - Device-side anomalies (a KV row outside the cache, a frontier wider than max_active,
+ *     a field length outside its slot) never fault: the offending item is clamped or
+ *     skipped and a sticky bit is set in the plan's status word (fdc_status).
+ *   - A plan is bound to the CUDA device that was current in fdc_plan_graph.
+ */
+#ifndef FDC_H_
+#define FDC_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define FDC_MAX_NODES   64   /* fields per template (one 64-bit word per node set)          */
+#define FDC_TILE_ROWS   64   /* KV rows per tile of the visited-tile list                   */
+#define FDC_MAX_QROWS   128  /* max_active * (hq / hkv): query rows served by one KV read   */
+#define FDC_MAX_BATCH   4096 /* scenes per call                                             */
+
+enum {
+    FDC_OK            =  0,
+    FDC_ERR_NULL      = -1,  /* a required pointer is NULL                                  */
+    FDC_ERR_CYCLE     = -2,  /* the dependency graph has a directed cycle or a self loop    */
+    FDC_ERR_RANGE     = -3,  /* node id, node count, slot, n_fixed, max_active, layer, batch out of range */
+    FDC_ERR_SHAPE     = -4,  /* hq % hkv, head_dim not in {64,128}, rows < P+T, too many query rows, strides */
+    FDC_ERR_DTYPE     = -5,  /* dtype is neither FDC_F32 nor FDC_BF16                       */
+    FDC_ERR_WORKSPACE = -6,  /* workspace missing, misaligned or smaller than required      */
+    FDC_ERR_CUDA      = -7,  /* a CUDA runtime call failed (see fdc_last_cuda_error)        */
+    FDC_ERR_DEVICE    = -8   /* fdc_status: the device recorded an anomaly                  */
+};
+
+enum { FDC_F32 = 0, FDC_BF16 = 1 };
+
+/* bits of the sticky device status word */
+enum {
+    FDC_DEV_ROW_RANGE     = 1,  /* fdc_kv_append: kv_row outside [0, rows): row skipped      */
+    FDC_DEV_FRONTIER_WIDE = 2,  /* fdc_frontier: more ready fields than max_active: clamped, */
+                                /* the others wait for a later pass                          */
+    FDC_DEV_LEN_RANGE     = 4   /* fdc_state_init: a length outside [n_fixed+1, C]: clamped  */
+};
+
+typedef struct fdc_plan fdc_plan;
+
+/* Template description (Sec. 3.1-3.2).  All pointers are HOST memory, read during the call. */
+typedef struct {
+    int32_t        n_nodes;     /* fields, 1..FDC_MAX_NODES; node id = template order        */
+    int32_t        n_edges;
+    const int32_t* edges;       /* [n_edges][2] = (src, dst): dst needs src complete          */
+    const int32_t* slot_cap;    /* [n_nodes] C[v] >= 1: rows reserved for field v (Sec. 3.3) */
+    const int32_t* n_fixed;     /* [n_nodes] pre-filled field-name rows at the head of each  */
+                                /* slot (0 <= n_fixed < C), or NULL for none                  */
+    int32_t        prefix_len;  /* P >= 0: shared vision+prompt rows, visible to everyone    */
+    int32_t        max_active;  /* branch slots per scene per pass, 1..FDC_MAX_NODES         */
+} fdc_graph_desc;
+
+/* KV cache view.  k and v are DEVICE pointers to element [scene 0][layer 0][head 0][row 0][0];
+ * strides are in ELEMENTS; head_dim elements of a row are contiguous.  Row r of a scene is
+ * the prefix for r < P and template row r - P otherwise.  Required: every stride a multiple
+ * of 8 elements and k, v 16-byte aligned (128-bit accesses). */
+typedef struct {
+    void*   k;
+    void*   v;
+    int32_t dtype;              /* FDC_F32 | FDC_BF16 (also the dtype of q, k_new, v_new, out) */
+    int32_t batch, layers, hkv, hq, head_dim, rows;
+    int64_t stride_scene, stride_layer, stride_head, stride_row;
+} fdc_kv_desc;
+
+/* Sizes of the caller-owned buffers for `batch` scenes. */
+typedef struct {
+    int32_t cot_rows;           /* T = sum of C[v]                                            */
+    int32_t mask_words;         /* W = ceil(T / 64) words per branch bitmap                   */
+    int32_t ntile_max;          /* entries per scene of the tile list = ceil((P+T)/64)        */
+    int32_t max_active;
+    size_t  state_bytes;        /* d_state                                                    */
+    size_t  mask_bytes;         /* d_mask  : uint64 [batch][max_active][W]                    */
+    size_t  umask_bytes;        /* d_umask : uint64 [batch][W]                                */
+    size_t  tiles_bytes;        /* d_tiles : int32  [batch][ntile_max]                        */
+} fdc_sizes;
+
+/* Sec. 3.2 (the dependency graph) and Eq. 1.  Validates the template (ids in range, no
+ * cycle), builds on the host the parent sets, successor lists, the ANCESTOR set of every
+ * node (transitive closure of E: bit u of anc[v] <=> a path u -> ... -> v) and the slot
+ * bases base[v] = sum_{u<v} C[u], and copies them to the current device.  Host call;
+ * allocates the plan (a few KB of device memory); synchronises.  *out is set on success. */
+int fdc_plan_graph(const fdc_graph_desc* desc, fdc_plan** out);
+int fdc_plan_destroy(fdc_plan* plan);
+
+int fdc_plan_query(const fdc_plan* plan, int32_t batch, fdc_sizes* out);
+
+/* Host copies of the plan's tables, for inspection and tests: anc/par uint64 [n],
+ * base int32 [n+1], indegree int32 [n].  Any output pointer may be NULL. */
+int fdc_plan_tables(const fdc_plan* plan, uint64_t* anc, uint64_t* par, int32_t* base, int32_t* indegree);
+
+/* Sec. 3.2: the minimum number of forward passes = the largest cumulative number of
+ * generated tokens along any dependency chain.  len is HOST int32 [n] (rows of each field
+ * including its fixed ones); finish (HOST int32 [n], may be NULL) receives the 1-based pass in
+ * which each field emits its last token.  Host-only arithmetic. */
+int fdc_plan_critical_path(const fdc_plan* plan, const int32_t* len, int32_t* steps, int32_t* finish);
+
+/* Algorithm 1 initialisation for `batch` scenes: d_v = indegree, S = sources, no field has
+ * generated anything (tok[v] = n_fixed[v]).  d_len: DEVICE int32 [batch][n] = the number of
+ * rows after which field v of scene s is finished when no finish flag arrives earlier
+ * (synthetic runs: the field's true length), or NULL to use the slot C[v] (truncation to the
+ * fixed length, Sec. 3.3).  Values are clamped to [n_fixed+1, C]. */
+int fdc_state_init(const fdc_plan* plan, int32_t batch, const int32_t* d_len, void* d_state, void* stream);
+
+/* Algorithm 1, one loop iteration (Sec. 3.2).  First retires the fields of the previous pass
+ * that finished - branch slot b of scene s is finished if d_finish[s][b] != 0 (DEVICE uint8
+ * [batch][max_active], e.g. "end of field sampled"; may be NULL) or its row count reached its
+ * limit - lowers d_u of their successors and admits those that reach 0.  Then emits the packed
+ * list of this pass, one entry per ready field in ascending node id:
+ *   d_n_active int32 [batch]               A = ready fields (<= max_active)
+ *   d_node     int32 [batch][max_active]   field id, -1 in unused slots
+ *   d_tok_idx  int32 [batch][max_active]   t: index within the slot of the token decoded now
+ *   d_kv_row   int32 [batch][max_active]   P + base[v] + t (Sec. 3.3: fixed slots), -1 unused
+ *   d_pos_id   int32 [batch][max_active]   the same value: position id = reserved row
+ *   d_all_done int32 [1]                   1 iff no scene has a ready field left
+ * A field admitted in this call decodes its first token in this pass; a field that finishes
+ * in this pass is retired by the NEXT call.  All outputs are DEVICE memory. */
+int fdc_frontier(const fdc_plan* plan, int32_t batch, void* d_state, const uint8_t* d_finish,
+                 int32_t* d_n_active, int32_t* d_node, int32_t* d_tok_idx, int32_t* d_kv_row,
+                 int32_t* d_pos_id, int32_t* d_all_done, void* stream);
+
+/* Eq. 1 + Sec. 3.3 as bitmaps, for the pass fdc_frontier just emitted (reads d_state).
+ *   d_mask  uint64 [batch][max_active][W]  bit i of word w <=> template row 64w+i is visible
+ *           to that branch: a real (non-padding) row of an ancestor field, a row <= t of its
+ *           own field, or a fixed field-name row at a lower position.  Unused slots: 0.
+ *           Prefix rows are not in the bitmap: they are visible to every branch.
+ *   d_umask uint64 [batch][W]              OR over the scene's branches
+ *   d_tiles int32  [batch][ntile_max], d_ntiles int32 [batch]
+ *           ascending ids of the KV tiles (rows 64i..64i+63 of the scene's cache, prefix
+ *           included) holding at least one row visible to some branch; 0 tiles for a scene
+ *           with no active branch. */
+int fdc_build_masks(const fdc_plan* plan, int32_t batch, const void* d_state, uint64_t* d_mask,
+                    uint64_t* d_umask, int32_t* d_tiles, int32_t* d_ntiles, void* stream);
+
+/* Sec. 3.3 (shared KV cache, reused by all later passes): for every scene s and branch
+ * b < d_n_active[s], copy d_k_new/d_v_new [batch][max_active][hkv][head_dim] into cache row
+ * d_kv_row[s][b] of `layer`.  Padding rows are never written.  Rows outside [0, rows) are
+ * skipped and flagged in the plan's status word. */
+int fdc_kv_append(const fdc_plan* plan, const fdc_kv_desc* kv, int32_t layer, const int32_t* d_n_active,
+                  const int32_t* d_kv_row, const void* d_k_new, const void* d_v_new, void* stream);
+
+/* Scratch for fdc_decode_attn (split partials); depends on the plan, the cache shape and the
+ * device's SM count. */
+int fdc_attn_workspace_bytes(const fdc_plan* plan, const fdc_kv_desc* kv, size_t* bytes);
+
+/* The masked attention of one layer for the pass described by d_n_active/d_mask/d_tiles
+ * (Sec. 3.3): for scene s, branch b < A, query head h (KV head h / (hq/hkv)),
+ *     out = softmax_r(scale * q . K[r]) V[r]   over the rows r visible to branch b
+ * (prefix rows and the rows set in d_mask[s][b]).  q and out: DEVICE [batch][max_active][hq]
+ * [head_dim] in the cache dtype; rows of unused branch slots are not touched.  Scores,
+ * softmax and accumulation are fp32; bf16 output is rounded to nearest even.  Each visited
+ * KV tile is read once for all branches and all heads of its KV group; invisible K/V rows
+ * may hold anything (NaN included).  d_workspace: DEVICE, 256-byte aligned,
+ * >= fdc_attn_workspace_bytes; its contents are undefined afterwards. */
+int fdc_decode_attn(const fdc_plan* plan, const fdc_kv_desc* kv, int32_t layer, const int32_t* d_n_active,
+                    const uint64_t* d_mask, const int32_t* d_tiles, const int32_t* d_ntiles,
+                    const void* d_q, void* d_out, float scale, void* d_workspace, size_t ws_bytes,
+                    void* stream);
+
+/* Reads (and with clear != 0 resets) the sticky device status word after synchronising
+ * `stream`.  *host_bits receives the FDC_DEV_* bits; returns FDC_ERR_DEVICE if non-zero. */
+int fdc_status(const fdc_plan* plan, int32_t* host_bits, int32_t clear, void* stream);
+
+/* Selects the attention kernel: 0 = automatic, 1 = CUDA-core reference kernel (any dtype),
+ * other values as listed by fdc_kernel_name.  Unsupported combinations fall back to 1. */
+int fdc_set_attn_kernel(fdc_plan* plan, int32_t which);
+const char* fdc_kernel_name(int32_t which);
+
+/* Number of kernels this library has launched in the calling process so far. */
+int64_t fdc_launch_count(void);
+
+const char* fdc_strerror(int code);
+const char* fdc_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FDC_H_ */

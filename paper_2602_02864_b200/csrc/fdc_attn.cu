@@ -1,0 +1,98 @@
+// fdc_decode_attn: argument checks, kernel selection, split pass + combine pass.
+#include <cmath>
+
+#include "fdc_internal.h"
+
+using namespace fdc;
+
+namespace {
+
+// Upper bound of split CTAs any kernel variant uses (2 per SM), so that the workspace size
+// does not depend on the variant.
+inline int max_ctas(const fdc_plan* p) { return 2 * p->sm_count; }
+
+inline size_t ws_bytes_for(const fdc_plan* p, const fdc_kv_desc* kv)
+{
+    const size_t slots = (size_t)max_ctas(p) + (size_t)kv->batch * kv->hkv;
+    const size_t mmax = (size_t)p->h.max_active * (kv->hq / kv->hkv);
+    size_t b = slots * mmax * (kv->head_dim + 2) * sizeof(float);
+    return (b + 255) & ~(size_t)255;
+}
+
+}  // namespace
+
+extern "C" {
+
+int fdc_attn_workspace_bytes(const fdc_plan* p, const fdc_kv_desc* kv, size_t* bytes)
+{
+    if (!bytes) return FDC_ERR_NULL;
+    int rc = check_kv_desc(p, kv, 0);
+    if (rc) return rc;
+    *bytes = ws_bytes_for(p, kv);
+    return FDC_OK;
+}
+
+int fdc_set_attn_kernel(fdc_plan* p, int32_t which)
+{
+    if (!p) return FDC_ERR_NULL;
+    if (which < 0 || which > 1) return FDC_ERR_RANGE;
+    p->attn_kernel = which;
+    return FDC_OK;
+}
+
+const char* fdc_kernel_name(int32_t which)
+{
+    switch (which) {
+        case 0: return "auto";
+        case 1: return "ref_cuda_core";
+        default: return nullptr;
+    }
+}
+
+int fdc_decode_attn(const fdc_plan* p, const fdc_kv_desc* kv, int32_t layer, const int32_t* d_n_active,
+                    const uint64_t* d_mask, const int32_t* d_tiles, const int32_t* d_ntiles, const void* d_q,
+                    void* d_out, float scale, void* d_workspace, size_t ws_bytes, void* stream)
+{
+    int rc = check_kv_desc(p, kv, layer);
+    if (rc) return rc;
+    if (!d_n_active || !d_mask || !d_tiles || !d_ntiles || !d_q || !d_out) return FDC_ERR_NULL;
+    if (!d_workspace || ((uintptr_t)d_workspace & 255) || ws_bytes < ws_bytes_for(p, kv)) return FDC_ERR_WORKSPACE;
+    if (((uintptr_t)d_q & 15) || ((uintptr_t)d_out & 15)) return FDC_ERR_SHAPE;
+    if (!(scale > 0.f) || !std::isfinite(scale)) return FDC_ERR_RANGE;
+    const int es = kv->dtype == FDC_F32 ? 4 : 2;
+
+    AttnParams a;
+    a.k = (const char*)kv->k + (size_t)layer * kv->stride_layer * es;
+    a.v = (const char*)kv->v + (size_t)layer * kv->stride_layer * es;
+    a.stride_scene = kv->stride_scene;
+    a.stride_head = kv->stride_head;
+    a.stride_row = kv->stride_row;
+    a.q = d_q;
+    a.out = d_out;
+    a.mask = d_mask;
+    a.tiles = d_tiles;
+    a.ntiles = d_ntiles;
+    a.n_active = d_n_active;
+    a.batch = kv->batch;
+    a.hkv = kv->hkv;
+    a.hq = kv->hq;
+    a.group = kv->hq / kv->hkv;
+    a.max_active = p->h.max_active;
+    a.mmax = a.max_active * a.group;
+    a.W = p->h.W;
+    a.P = p->h.P;
+    a.rows = kv->rows;
+    a.ntile_max = p->h.ntile_max;
+    a.scale_log2 = scale * 1.4426950408889634f;
+    const size_t slots = (size_t)max_ctas(p) + (size_t)kv->batch * kv->hkv;
+    a.ws_o = (float*)d_workspace;
+    a.ws_ml = a.ws_o + slots * a.mmax * kv->head_dim;
+    a.n_cta = p->sm_count;
+
+    cudaStream_t st = (cudaStream_t)stream;
+    rc = launch_attn_ref(a, kv->dtype, kv->head_dim, st);
+    if (rc) return rc;
+    return launch_attn_combine(a, kv->dtype, kv->head_dim, st);
+}
+
+}  // extern "C"

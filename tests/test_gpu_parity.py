@@ -1,0 +1,167 @@
+"""GPU parity: the C-ABI CUDA path against the CPU checker on the same seeded inputs.
+Integers (schedule, slots, positions, bitmaps, tile lists, cache contents) bit-exact;
+attention within the stated tolerances."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2602_02864_b200 import workloads as wl
+
+from harness import run_and_compare
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    from paper_2602_02864_b200 import build
+    build.build()
+
+
+def test_cfg0_tiny_every_step():
+    w = wl.cfg0_tiny()
+    r = run_and_compare(w)
+    assert r["steps"] == 48 and r["checked"] == 96 * 4
+
+
+def test_cfg0_tiny_bf16_head128():
+    w = wl.cfg0_tiny()
+    w.dtype, w.head_dim = "bf16", 128
+    run_and_compare(w)
+
+
+def test_cfg1_7b_reduced_layers():
+    """Config 1 shapes (28 q heads / 4 KV heads -> group 7, prefix 2048), 2 of its layers."""
+    w = wl.cfg1_7b(layers=2)
+    n = int(w.lens[0, :6].max() + w.lens[0, 6] + w.lens[0, 7])
+    steps = set(range(0, n, 9)) | {int(w.lens[0, :6].min()) - 1, int(w.lens[0, :6].min()),
+                                   int(w.lens[0, :6].max()) - 1, int(w.lens[0, :6].max()), n - 1}
+    r = run_and_compare(w, check_steps=steps)
+    assert r["steps"] == n
+
+
+def test_cfg2_batched_reduced():
+    """Config 2 shapes with 4 of its 16 scenes and 1 layer: scenes in different phases."""
+    w = wl.cfg2_batched(layers=1, batch=4)
+    r = run_and_compare(w, check_steps=set(range(0, 300, 17)) | {15, 16, 95, 96})
+    assert r["checked"] > 0
+
+
+def test_cfg3_wide_reduced():
+    """Config 3 shapes (16-wide frontier, 64 query rows per KV head), 2 scenes, 1 layer."""
+    w = wl.cfg3_wide(layers=1, batch=2)
+    r = run_and_compare(w, check_steps={0, 1, 47, 48, 49, 95, 96, 143})
+    assert r["steps"] == 144
+
+
+@pytest.mark.parametrize("branches,chain", [(1, False), (4, False), (32, False), (4, True)])
+def test_cfg4_sweep_points_small_prefix(branches, chain):
+    w = wl.cfg4_sweep(1024, branches, 2, chain=chain)
+    r = run_and_compare(w, check_steps={0, 1, 31, 63, 64, 255})
+    assert r["steps"] == (64 * branches if chain else 64)
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_random_templates_with_fixed_tokens_and_ragged_prefix(seed):
+    """Random DAGs, ragged slots, fixed field-name rows, prefix lengths that are not tile
+    multiples (including 0), caches longer than P+T, several scenes."""
+    w = wl.random_template(3000 + seed, n_nodes=3 + seed, edge_prob=0.3, cap_lo=2, cap_hi=70, batch=3,
+                           prefix_len=[0, 1, 63, 64, 65, 130, 200, 7, 128, 31, 96, 5][seed], fixed_hi=seed % 4,
+                           hq=8, hkv=2, head_dim=64 if seed % 2 else 128, dtype="f32" if seed % 3 else "bf16")
+    w.max_active = w.n_nodes
+    run_and_compare(w, extra_rows=seed * 5)
+
+
+def test_finish_flags_drive_the_schedule():
+    w = wl.random_template(4242, n_nodes=9, edge_prob=0.3, cap_hi=20, batch=4, prefix_len=70)
+    run_and_compare(w, use_finish_flags=True)
+
+
+def test_truncation_to_slot_when_no_length_given():
+    """Without lengths or flags every field runs to its slot capacity (Sec. 3.3: truncate)."""
+    w = wl.random_template(4243, n_nodes=6, edge_prob=0.4, cap_hi=12, batch=2, prefix_len=10)
+    w.lens = np.tile(np.array(w.slot_cap, np.int32), (2, 1))
+    from paper_2602_02864_b200 import fdc
+    from harness import make_oracle, compare_int_tables
+    oracle = make_oracle(w)
+    sess = fdc.DecodeSession(w.n_nodes, w.edges, w.slot_cap, w.n_fixed, w.prefix_len, w.max_active, w.batch)
+    sess.init(None)
+    for step in range(oracle.n_steps):
+        sess.frontier(None)
+        sess.build_masks()
+        compare_int_tables(sess, oracle, step)
+    sess.frontier(None)
+    assert int(sess.all_done.item()) == 1
+
+
+def test_device_anomalies_are_flagged_not_fatal():
+    from paper_2602_02864_b200 import fdc
+    # frontier wider than max_active: clamped, flagged, and the run still completes correctly
+    sess = fdc.DecodeSession(4, [], [3, 3, 3, 3], None, 4, 2, 1)
+    sess.init(None)
+    seen = []
+    for _ in range(20):
+        sess.frontier(None)
+        if int(sess.all_done.item()):
+            break
+        seen.append(sess.node[0, :int(sess.n_active.item())].tolist())
+    assert seen == [[0, 1]] * 3 + [[2, 3]] * 3
+    assert sess.status(clear=True) == fdc.FDC_DEV_FRONTIER_WIDE
+    assert sess.status() == 0
+    # lengths outside the slot are clamped and flagged
+    sess.init(torch.tensor([[9, 0, 2, 3]], dtype=torch.int32, device="cuda"))
+    assert sess.status(clear=True) == fdc.FDC_DEV_LEN_RANGE
+    # a KV row outside the cache is skipped and flagged
+    k = torch.zeros(1, 1, 1, 16, 64, device="cuda")
+    v = torch.zeros_like(k)
+    sess.bind_cache(k, v, 1)
+    sess.frontier(None)
+    sess.kv_row.fill_(99)
+    kn = torch.ones(1, 2, 1, 64, device="cuda")
+    sess.kv_append(0, kn, kn)
+    # (the 4-wide frontier was clamped to 2 again, so that bit is set too)
+    assert sess.status(clear=True) == fdc.FDC_DEV_ROW_RANGE | fdc.FDC_DEV_FRONTIER_WIDE
+    assert float(k.abs().sum()) == 0.0
+    sess.close()
+
+
+def test_argument_errors():
+    from paper_2602_02864_b200 import fdc
+    sess = fdc.DecodeSession(2, [(0, 1)], [4, 4], None, 8, 1, 1)
+    k = torch.zeros(1, 1, 2, 16, 64, device="cuda")
+    with pytest.raises(fdc.FdcError) as e:
+        sess.bind_cache(k, k.clone(), 3)                # hq % hkv
+    assert e.value.code == fdc.FDC_ERR_SHAPE
+    k = torch.zeros(1, 1, 2, 15, 64, device="cuda")      # rows < P + T
+    with pytest.raises(fdc.FdcError) as e:
+        sess.bind_cache(k, k.clone(), 2)
+    assert e.value.code == fdc.FDC_ERR_SHAPE
+    k = torch.zeros(1, 1, 2, 16, 64, device="cuda")
+    sess.bind_cache(k, k.clone(), 2)
+    q = torch.zeros(1, 1, 2, 64, device="cuda")
+    with pytest.raises(fdc.FdcError) as e:
+        fdc.fdc_decode_attn(sess.plan, sess.kv, 0, sess.n_active, sess.mask, sess.tiles, sess.ntiles, q, q.clone(),
+                            0.125, sess.workspace, 16)
+    assert e.value.code == fdc.FDC_ERR_WORKSPACE
+    with pytest.raises(fdc.FdcError) as e:
+        sess.kv_append(3, q, q)
+    assert e.value.code == fdc.FDC_ERR_RANGE
+    sess.close()
+
+
+def test_critical_path_host_call_matches_device_schedule():
+    from paper_2602_02864_b200 import fdc
+    from oracle import schedule as sch
+    for seed in range(10):
+        w = wl.random_template(8800 + seed, n_nodes=4 + seed, fixed_hi=2)
+        plan = fdc.fdc_plan_graph(w.n_nodes, w.edges, w.slot_cap, w.n_fixed, w.prefix_len, w.max_active)
+        steps, fin = fdc.fdc_plan_critical_path(plan, w.lens[0])
+        passes = sch.simulate(w.n_nodes, w.edges, w.lens[0].tolist(), w.n_fixed)
+        assert steps == len(passes)
+        anc, par, base, indeg = fdc.fdc_plan_tables(plan, w.n_nodes)
+        ref_anc = sch.ancestors(w.n_nodes, w.edges)
+        for v in range(w.n_nodes):
+            assert {u for u in range(w.n_nodes) if int(anc[v]) >> u & 1} == ref_anc[v]
+            assert fin[v] == 1 + max(k for k, p in enumerate(passes) if any(x == v for x, _ in p))
+        assert base.tolist() == sch.slot_base(w.slot_cap)
+        fdc.fdc_plan_destroy(plan)
