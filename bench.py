@@ -1,0 +1,423 @@
+#!/usr/bin/env python
+"""Benchmark of the dependency-masked parallel-decoding step on B200.
+
+One "step" = one forward pass of the whole hot path for one batch of scenes:
+fdc_frontier -> fdc_build_masks -> for every layer: fdc_kv_append -> fdc_decode_attn
+(split-KV pass + combine pass).  The metric is achieved KV-cache bandwidth: the bytes the
+method itself must move per step (every KV row visible to some branch read once for all
+branches and GQA heads, plus q, out, the appended rows and the bitmaps) divided by the
+step time.  Prints ONE JSON line on stdout (rank 0).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2|cfg1|cfg3|cfg0]
+                  [--impl fdc|reference] [--no-also]
+Under torchrun (N > 1) every rank runs an independent replica of the workload (scenes shard
+with no exchange): weak scaling, time = max over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "masked_decode_attn_kv_bandwidth"
+UNIT = "GB/s"
+NOMINAL_HBM_GBS = 8000.0
+
+
+def log(*a):
+    print(*a, file=sys.stderr, flush=True)
+
+
+def get_workload(name: str):
+    from paper_2602_02864_b200 import workloads as wl
+    return {"cfg0": wl.cfg0_tiny, "cfg1": wl.cfg1_7b, "cfg2": wl.cfg2_batched, "cfg3": wl.cfg3_wide}[name]()
+
+
+WORKLOAD_TEXT = {
+    "cfg0": "configs[0] tiny fp32: 1 layer, 4q/2kv heads, D 64, batch 1, prefix 256, 6-field DAG, 16-token slots",
+    "cfg1": "configs[1] 7B-class bf16: 28 layers, 28q/4kv heads, D 128, batch 1, prefix 2048, 8-field DAG, slots 64 (len U32-64)",
+    "cfg2": "configs[2] batched scenes bf16: 32 layers, 32q/8kv heads, D 128, batch 16, prefix 4096, 8-field DAG, slots 96 (len U16-96 per scene)",
+    "cfg3": "configs[3] wide graph bf16: 32 layers, 32q/8kv heads, D 128, batch 8, prefix 8192, 16 leaves -> 2 aggregators -> final, 48-token slots",
+}
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return float(d["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    return 6650.0, "fallback (6.65 TB/s, earlier measurement on this pool)"
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs (read only)."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc = index, None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, mx, reasons, pw = [], [], set(), []
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0]))
+                mx.append(float(f[1]))
+                pw.append(float(f[2]))
+            except ValueError:
+                continue
+            for n, val in zip(names, f[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "power_w_max": max(pw) if pw else None, "samples": len(sm), "reasons": sorted(reasons)}
+
+
+class StepBench:
+    """Device-resident state of one workload and the per-step launch sequence."""
+
+    def __init__(self, w, n_steps: int, device, seed_shift: int = 0):
+        import torch
+        from paper_2602_02864_b200 import fdc, workloads as wl
+        self.torch, self.fdc, self.w, self.device = torch, fdc, w, device
+        self.n_steps = n_steps
+        self.sess = fdc.DecodeSession(w.n_nodes, w.edges, w.slot_cap, w.n_fixed, w.prefix_len, w.max_active, w.batch,
+                                      device)
+        shape = (w.batch, w.layers, w.hkv, w.rows, w.head_dim)
+        self.k = torch.zeros(shape, dtype=w.torch_dtype, device=device)   # padding rows stay zero
+        self.v = torch.zeros(shape, dtype=w.torch_dtype, device=device)
+        g = torch.Generator(device=device)
+        g.manual_seed(w.seed + 7919 * seed_shift)
+        for l in range(w.layers):                                          # prefix KV, in HBM before timing
+            for t in (self.k, self.v):
+                t[:, l, :, :w.prefix_len] = (torch.randn((w.batch, w.hkv, w.prefix_len, w.head_dim), generator=g,
+                                                         device=device) * w.kv_scale).to(w.torch_dtype)
+        self.sess.bind_cache(self.k, self.v, w.hq)
+        self.lens = torch.from_numpy(w.lens).to(device)
+        qs = (n_steps, w.layers, w.batch, w.max_active, w.hq, w.head_dim)
+        ks = (n_steps, w.layers, w.batch, w.max_active, w.hkv, w.head_dim)
+        self.q = torch.randn(qs, generator=g, device=device).to(w.torch_dtype)
+        self.kn = (torch.randn(ks, generator=g, device=device) * w.kv_scale).to(w.torch_dtype)
+        self.vn = (torch.randn(ks, generator=g, device=device) * w.kv_scale).to(w.torch_dtype)
+        self.out = torch.zeros((w.layers, w.batch, w.max_active, w.hq, w.head_dim), dtype=w.torch_dtype, device=device)
+        self.umask_log = torch.zeros((n_steps,) + tuple(self.sess.umask.shape), dtype=torch.int64, device=device)
+        self.nact_log = torch.zeros((n_steps, w.batch), dtype=torch.int32, device=device)
+        self.launches_per_step = 2 + 3 * w.layers
+
+    def reset(self):
+        self.sess.init(self.lens)
+
+    def step(self, i: int, q=None, kn=None, vn=None, log_masks: bool = False):
+        s, w = self.sess, self.w
+        q = self.q[i] if q is None else q
+        kn = self.kn[i] if kn is None else kn
+        vn = self.vn[i] if vn is None else vn
+        s.frontier(None)
+        s.build_masks()
+        if log_masks:
+            self.umask_log[i].copy_(s.umask)
+            self.nact_log[i].copy_(s.n_active)
+        for l in range(w.layers):
+            s.kv_append(l, kn[l], vn[l])
+            s.decode_attn(l, q[l], self.out[l], w.softmax_scale)
+
+    # ---- the method's own traffic (what one launch / one step must move) ----
+    def algorithmic_bytes(self, steps):
+        """Per step in `steps`: bytes of one layer-step, from the logged union bitmaps."""
+        w = self.w
+        um = self.umask_log.cpu().numpy().view(np.uint64)
+        na = self.nact_log.cpu().numpy()
+        row_bytes = 2 * w.hkv * w.head_dim * w.esize
+        per = []
+        for i in steps:
+            b = 0
+            for s in range(w.batch):
+                A = int(na[i, s])
+                if A == 0:
+                    continue
+                vis_rows = w.prefix_len + sum(bin(int(x)).count("1") for x in um[i, s])
+                b += vis_rows * row_bytes                               # each visible KV row once
+                b += 2 * A * w.hq * w.head_dim * w.esize                # q in, out
+                b += A * row_bytes                                      # appended rows
+                b += A * um.shape[2] * 8                                # bitmaps
+            per.append(b)
+        return per
+
+
+def run_fdc(args, rank: int, world: int):
+    import torch
+    import torch.distributed as dist
+    from paper_2602_02864_b200 import build as _build
+    if rank == 0:
+        _build.build()
+    if world > 1:
+        dist.barrier()
+    from paper_2602_02864_b200 import fdc
+    local = int(os.environ.get("LOCAL_RANK", 0))
+    torch.cuda.set_device(local)
+    device = torch.device("cuda", local)
+    peak, peak_src = measured_peaks()
+
+    def measure(name: str, K: int, W: int, with_e2e: bool, sample_clocks: bool):
+        w = get_workload(name)
+        total = W + K
+        sb = StepBench(w, total, device, seed_shift=rank)
+        ev = lambda: torch.cuda.Event(enable_timing=True)  # noqa: E731
+        stream = torch.cuda.current_stream()
+
+        # pass 0: untimed, logs the bitmaps so that the algorithmic bytes are known; also a warm-up
+        sb.reset()
+        for i in range(total):
+            sb.step(i, log_masks=True)
+        torch.cuda.synchronize()
+        per_layer_bytes = sb.algorithmic_bytes(range(total))
+        step_bytes = [b * w.layers for b in per_layer_bytes]
+        timed_bytes = sum(step_bytes[W:])
+        status = sb.sess.status(clear=True)
+
+        # pass 1 (the number): W warm-up steps, then exactly K timed steps, device-resident inputs
+        sampler = ClockSampler(local)
+        sb.reset()
+        for i in range(W):
+            sb.step(i)
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+        if sample_clocks:
+            sampler.start()
+        l0 = fdc.fdc_launch_count()
+        e0, e1 = ev(), ev()
+        e0.record(stream)
+        for i in range(W, total):
+            sb.step(i)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        launches = fdc.fdc_launch_count() - l0
+        clocks = sampler.stop() if sample_clocks else None
+        ms = e0.elapsed_time(e1)
+        if world > 1:
+            t = torch.tensor([ms], device=device, dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+            dist.barrier()
+
+        # pass 2: per-launch duration of the dominant kernel (split-KV pass), CUDA events recorded by
+        # the library itself on the launching stream around every such launch of the same K steps
+        sb.reset()
+        for i in range(W):
+            sb.step(i)
+        torch.cuda.synchronize()
+        fdc.fdc_profile(sb.sess.plan, True)
+        for i in range(W, total):
+            sb.step(i)
+        prof = fdc.fdc_profile_read(sb.sess.plan)
+        fdc.fdc_profile(sb.sess.plan, False)
+        split_ms, split_n = prof["split_ms"], prof["split_launches"]
+        comb_ms = prof["combine_ms"]
+        roof = None
+        if split_n:
+            avg_bytes = timed_bytes / split_n
+            achieved = avg_bytes / (split_ms / split_n * 1e-3) / 1e9
+            roof = {"kernel": prof["kernel"], "bound": "hbm", "achieved": round(achieved, 1), "peak": peak,
+                    "unit": "GB/s", "frac": round(achieved / peak, 4), "peak_source": peak_src,
+                    "traffic": None, "launches": split_n, "avg_launch_us": round(split_ms / split_n * 1e3, 2),
+                    "algorithmic_bytes_per_launch": int(avg_bytes),
+                    "combine_avg_launch_us": round(comb_ms / split_n * 1e3, 2),
+                    "frac_of_nominal_8TBs": round(achieved / NOMINAL_HBM_GBS, 4)}
+
+        # pass 3: end to end through the C ABI with HOST buffers: every step copies its q / k_new /
+        # v_new from pinned host memory and reads the step's attention output back
+        e2e = None
+        if with_e2e:
+            hq_ = sb.q[W:].cpu().pin_memory()
+            hk_ = sb.kn[W:].cpu().pin_memory()
+            hv_ = sb.vn[W:].cpu().pin_memory()
+            hout = torch.empty_like(sb.out, device="cpu").pin_memory()
+            dq, dk, dv = torch.empty_like(sb.q[0]), torch.empty_like(sb.kn[0]), torch.empty_like(sb.vn[0])
+            sb.reset()
+            for i in range(W):
+                sb.step(i)
+            if world > 1:
+                dist.barrier()
+            torch.cuda.synchronize()
+            e0, e1 = ev(), ev()
+            e0.record(stream)
+            for i in range(K):
+                dq.copy_(hq_[i], non_blocking=True)
+                dk.copy_(hk_[i], non_blocking=True)
+                dv.copy_(hv_[i], non_blocking=True)
+                sb.step(W + i, dq, dk, dv)
+                hout.copy_(sb.out, non_blocking=True)
+            e1.record(stream)
+            torch.cuda.synchronize()
+            ems = e0.elapsed_time(e1)
+            if world > 1:
+                t = torch.tensor([ems], device=device, dtype=torch.float64)
+                dist.all_reduce(t, op=dist.ReduceOp.MAX)
+                ems = float(t.item())
+            h2d = (dq.numel() + dk.numel() + dv.numel()) * w.esize
+            d2h = sb.out.numel() * w.esize
+            e2e = {"value": round(world * timed_bytes / (ems * 1e-3) / 1e9, 1), "unit": UNIT,
+                   "ms_per_step": round(ems / K, 4), "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
+
+        value = world * timed_bytes / (ms * 1e-3) / 1e9
+        res = {"workload": name, "value": value, "ms": ms, "ms_per_step": ms / K, "launches": launches,
+               "roofline": roof, "e2e": e2e, "clocks": clocks, "status": status,
+               "step_us": round(ms / K * 1e3, 1), "layer_step_us": round(ms / K / w.layers * 1e3, 2),
+               "bytes_per_step": int(timed_bytes / K), "avg_active_per_scene": float(sb.nact_log[W:].float().mean()),
+               "pct_of_8TBs": round(100 * value / world / NOMINAL_HBM_GBS, 1),
+               "pct_of_measured_copy": round(100 * value / world / peak, 1)}
+        sb.sess.close()
+        del sb
+        torch.cuda.empty_cache()
+        return res, w
+
+    main, w = measure(args.workload, args.steps, args.warmup, True, True)
+    also = {}
+    if not args.no_also and world == 1:
+        for other in ("cfg1", "cfg3"):
+            if other == args.workload:
+                continue
+            r, _ = measure(other, min(args.steps, 20), max(3, min(args.warmup, 5)), False, False)
+            also[other] = {k: (round(v, 2) if isinstance(v, float) else v) for k, v in r.items()
+                           if k in ("value", "step_us", "layer_step_us", "bytes_per_step", "pct_of_8TBs",
+                                    "pct_of_measured_copy", "roofline", "avg_active_per_scene")}
+            also[other]["workload"] = WORKLOAD_TEXT[other]
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu:
+        cpu = cpu_baseline(args.workload, budget_s=12.0)
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": round(main["value"], 1), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": round(main["ms_per_step"], 4), "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": w.dtype, "data": "synthetic",
+            "config": {"workload": WORKLOAD_TEXT[args.workload], "scenes_per_gpu": w.batch, "layers": w.layers,
+                       "l2": "inputs larger than L2: each layer reads its own KV buffer, %.1f GB of KV per step"
+                             % (main["bytes_per_step"] / 1e9),
+                       "parallelism": "replicas" if world > 1 else "1 GPU",
+                       "step": "frontier + build_masks + layers x (kv_append + decode_attn[split + combine])"},
+            "step_us": main["step_us"], "layer_step_us": main["layer_step_us"],
+            "bytes_per_step": main["bytes_per_step"], "avg_active_branches_per_scene": round(main["avg_active_per_scene"], 2),
+            "pct_of_8TBs": main["pct_of_8TBs"], "pct_of_measured_copy": main["pct_of_measured_copy"],
+            "roofline": main["roofline"], "cpu_baseline": cpu, "e2e": main["e2e"], "clocks": main["clocks"],
+            "gpu_launches": int(main["launches"]), "device_status": main["status"], "also": also,
+            "paper_context": "paper reports 3.1-4.1x CoT speedup end to end on 1x A100 80GB (bf16); no kernel-level number",
+        }
+        print(json.dumps(line), flush=True)
+
+
+def cpu_baseline(name: str, budget_s: float = 12.0, steps=None, warmup=0):
+    """The float64 CPU checker as it stands, timed on this machine's host cores on a bounded sample
+    of the workload: whole (scene, layer) attention calls at the first pass of the schedule
+    (widest frontier, prefix + first template rows visible)."""
+    import torch
+    from oracle import attention as oatt
+    from oracle import schedule as sch
+    from paper_2602_02864_b200 import workloads as wl
+    w = get_workload(name)
+    passes = sch.simulate(w.n_nodes, w.edges, w.lens[0].tolist(), w.n_fixed)
+    tab = sch.pass_tables(w.n_nodes, w.edges, w.slot_cap, w.lens[0].tolist(), w.n_fixed, w.prefix_len, passes[0])
+    A = len(passes[0])
+    g = torch.Generator().manual_seed(w.seed)
+    K = (torch.randn((w.hkv, w.rows, w.head_dim), generator=g) * w.kv_scale).to(w.torch_dtype).float().numpy()
+    V = (torch.randn((w.hkv, w.rows, w.head_dim), generator=g) * w.kv_scale).to(w.torch_dtype).float().numpy()
+    q = torch.randn((A, w.hq, w.head_dim), generator=g).to(w.torch_dtype).float().numpy()
+    row_bytes = 2 * w.hkv * w.head_dim * w.esize
+    vis_rows = int(tab["vis"].any(axis=0).sum())
+    call_bytes = vis_rows * row_bytes + 2 * A * w.hq * w.head_dim * w.esize + A * row_bytes + A * tab["mask"].shape[1] * 8
+    oatt.attention(q, K, V, tab["vis"], w.softmax_scale)            # builds/loads the library, warms caches
+    for _ in range(warmup):
+        oatt.attention(q, K, V, tab["vis"], w.softmax_scale)
+    n, t0 = 0, time.perf_counter()
+    while True:
+        oatt.attention(q, K, V, tab["vis"], w.softmax_scale)
+        n += 1
+        el = time.perf_counter() - t0
+        if (steps is not None and n >= steps) or (steps is None and el >= budget_s):
+            break
+    cores = int(oatt.attention.last_threads)
+    return {"value": round(n * call_bytes / el / 1e9, 4), "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"{n} (scene, layer) attention calls of {name} at the first pass ({A} branches x {w.hq} heads, "
+                      f"{vis_rows} visible rows), float64, {el:.1f} s",
+            "ms_per_call": round(el / n * 1e3, 2), "calls": n}
+
+
+def run_reference(args, rank: int):
+    """`--impl reference`: the CPU checker timed on the host cores; each step is one bounded sample."""
+    if rank != 0:
+        return
+    cb = cpu_baseline(args.workload, steps=args.steps, warmup=min(args.warmup, 2))
+    w = get_workload(args.workload)
+    line = {"impl": "reference", "metric": METRIC, "value": cb["value"], "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": cb["ms_per_call"], "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": WORKLOAD_TEXT[args.workload], "step": "one (scene, layer) attention call of the first pass",
+                       "scenes_per_gpu": w.batch, "layers": w.layers},
+            "cpu_baseline": cb, "e2e": {"value": cb["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=40)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--workload", default="cfg2", choices=["cfg0", "cfg1", "cfg2", "cfg3"])
+    ap.add_argument("--impl", default="fdc", choices=["fdc", "reference"])
+    ap.add_argument("--no-also", action="store_true", help="skip the short runs of the other configurations")
+    ap.add_argument("--no-cpu", action="store_true", help="skip the CPU baseline leg")
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", 0))
+    world = int(os.environ.get("WORLD_SIZE", 1))
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+    if args.warmup < 3:
+        args.warmup = 3
+    if world > 1:
+        import torch
+        import torch.distributed as dist
+        torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", 0)))
+        dist.init_process_group("nccl")
+    run_fdc(args, rank, world)
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

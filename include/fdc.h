@@ -197,6 +197,14 @@ int fdc_status(const fdc_plan* plan, int32_t* host_bits, int32_t clear, void* st
 int fdc_set_attn_kernel(fdc_plan* plan, int32_t which);
 const char* fdc_kernel_name(int32_t which);
 
+/* Instrumentation for benchmarks: while enabled, fdc_decode_attn records CUDA events on the
+ * launching stream before its split pass, between the passes and after its combine pass (not
+ * usable during stream capture).  fdc_profile_read waits for the recorded events, returns
+ * the summed durations in milliseconds and the number of recorded calls, and clears the
+ * records.  At most 16384 calls are recorded between two reads. */
+int fdc_profile(fdc_plan* plan, int32_t enable);
+int fdc_profile_read(fdc_plan* plan, float* split_ms, float* combine_ms, int32_t* calls);
+
 /* Number of kernels this library has launched in the calling process so far. */
 int64_t fdc_launch_count(void);
 

@@ -147,6 +147,7 @@ int fdc_plan_graph(const fdc_graph_desc* g, fdc_plan** out)
 int fdc_plan_destroy(fdc_plan* p)
 {
     if (!p) return FDC_ERR_NULL;
+    prof_destroy(p);
     if (p->d) cudaFree(p->d);
     if (p->d_status) cudaFree(p->d_status);
     free(p->succ_ptr);

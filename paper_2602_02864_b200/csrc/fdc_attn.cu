@@ -1,5 +1,6 @@
 // fdc_decode_attn: argument checks, kernel selection, split pass + combine pass.
 #include <cmath>
+#include <vector>
 
 #include "fdc_internal.h"
 
@@ -19,9 +20,64 @@ inline size_t ws_bytes_for(const fdc_plan* p, const fdc_kv_desc* kv)
     return (b + 255) & ~(size_t)255;
 }
 
+struct Prof {
+    std::vector<cudaEvent_t> ev;      // 3 per recorded call
+    size_t used = 0;                  // events handed out since the last read
+    static constexpr size_t kMaxCalls = 16384;
+    cudaEvent_t next()
+    {
+        if (used == ev.size()) {
+            cudaEvent_t e;
+            if (cudaEventCreate(&e) != cudaSuccess) return nullptr;
+            ev.push_back(e);
+        }
+        return ev[used++];
+    }
+};
+
 }  // namespace
 
+namespace fdc {
+void prof_destroy(fdc_plan* p)
+{
+    Prof* pr = (Prof*)p->prof;
+    if (!pr) return;
+    for (cudaEvent_t e : pr->ev) cudaEventDestroy(e);
+    delete pr;
+    p->prof = nullptr;
+}
+}  // namespace fdc
+
 extern "C" {
+
+int fdc_profile(fdc_plan* p, int32_t enable)
+{
+    if (!p) return FDC_ERR_NULL;
+    if (enable && !p->prof) p->prof = new Prof;
+    p->prof_on = enable != 0;
+    return FDC_OK;
+}
+
+int fdc_profile_read(fdc_plan* p, float* split_ms, float* combine_ms, int32_t* calls)
+{
+    if (!p || !split_ms || !combine_ms || !calls) return FDC_ERR_NULL;
+    *split_ms = *combine_ms = 0.f;
+    *calls = 0;
+    Prof* pr = (Prof*)p->prof;
+    if (!pr) return FDC_OK;
+    for (size_t i = 0; i + 2 < pr->used; i += 3) {
+        cudaError_t e = cudaEventSynchronize(pr->ev[i + 2]);
+        float a = 0.f, b = 0.f;
+        if (e == cudaSuccess) e = cudaEventElapsedTime(&a, pr->ev[i], pr->ev[i + 1]);
+        if (e == cudaSuccess) e = cudaEventElapsedTime(&b, pr->ev[i + 1], pr->ev[i + 2]);
+        if (e != cudaSuccess) return set_cuda_error(e);
+        *split_ms += a;
+        *combine_ms += b;
+        *calls += 1;
+    }
+    pr->used = 0;
+    return FDC_OK;
+}
 
 int fdc_attn_workspace_bytes(const fdc_plan* p, const fdc_kv_desc* kv, size_t* bytes)
 {
@@ -90,9 +146,22 @@ int fdc_decode_attn(const fdc_plan* p, const fdc_kv_desc* kv, int32_t layer, con
     a.n_cta = p->sm_count;
 
     cudaStream_t st = (cudaStream_t)stream;
+    Prof* pr = p->prof_on ? (Prof*)p->prof : nullptr;
+    if (pr && pr->used + 3 > 3 * Prof::kMaxCalls) pr = nullptr;
+    cudaEvent_t e0 = nullptr, e1 = nullptr, e2 = nullptr;
+    if (pr) {
+        e0 = pr->next();
+        e1 = pr->next();
+        e2 = pr->next();
+        if (!e0 || !e1 || !e2) return set_cuda_error(cudaErrorMemoryAllocation);
+        cudaEventRecord(e0, st);
+    }
     rc = launch_attn_ref(a, kv->dtype, kv->head_dim, st);
     if (rc) return rc;
-    return launch_attn_combine(a, kv->dtype, kv->head_dim, st);
+    if (pr) cudaEventRecord(e1, st);
+    rc = launch_attn_combine(a, kv->dtype, kv->head_dim, st);
+    if (pr) cudaEventRecord(e2, st);
+    return rc;
 }
 
 }  // extern "C"

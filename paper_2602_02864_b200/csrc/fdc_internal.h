@@ -43,6 +43,8 @@ struct fdc_plan {
     int           device;
     int           sm_count;
     int           attn_kernel;       // 0 auto
+    void*         prof;              // event records of fdc_profile (nullptr when never enabled)
+    int           prof_on;
     int32_t*      succ_ptr;          // host CSR successor lists (kept for inspection)
     int32_t*      succ;
 };
@@ -72,6 +74,7 @@ int  set_cuda_error(cudaError_t e);                  // records the message, ret
 
 int launch_attn_ref(const AttnParams& p, int dtype, int head_dim, cudaStream_t st);
 int launch_attn_combine(const AttnParams& p, int dtype, int head_dim, cudaStream_t st);
+void prof_destroy(fdc_plan* plan);
 int  check_kv_desc(const fdc_plan* plan, const fdc_kv_desc* kv, int32_t layer);
 
 // ----------------------------------------------------------------------------------

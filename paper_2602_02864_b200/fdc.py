@@ -69,6 +69,9 @@ _decode_attn = _sig("fdc_decode_attn", c_i32, c_vp, ctypes.POINTER(fdc_kv_desc),
 _status = _sig("fdc_status", c_i32, c_vp, ctypes.POINTER(c_i32), c_i32, c_vp)
 _set_attn_kernel = _sig("fdc_set_attn_kernel", c_i32, c_vp, c_i32)
 _kernel_name = _sig("fdc_kernel_name", ctypes.c_char_p, c_i32)
+_profile = _sig("fdc_profile", c_i32, c_vp, c_i32)
+_profile_read = _sig("fdc_profile_read", c_i32, c_vp, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_float),
+                     ctypes.POINTER(c_i32))
 _launch_count = _sig("fdc_launch_count", c_i64)
 _strerror = _sig("fdc_strerror", ctypes.c_char_p, c_i32)
 _last_cuda_error = _sig("fdc_last_cuda_error", ctypes.c_char_p)
@@ -199,6 +202,16 @@ def fdc_set_attn_kernel(plan, which: int) -> None:
 def fdc_kernel_name(which: int) -> Optional[str]:
     s = _kernel_name(which)
     return s.decode() if s else None
+
+
+def fdc_profile(plan, enable: bool) -> None:
+    _check(_profile(plan, int(enable)), "fdc_profile")
+
+
+def fdc_profile_read(plan) -> dict:
+    a, b, n = ctypes.c_float(), ctypes.c_float(), c_i32()
+    _check(_profile_read(plan, ctypes.byref(a), ctypes.byref(b), ctypes.byref(n)), "fdc_profile_read")
+    return {"split_ms": a.value, "combine_ms": b.value, "split_launches": n.value, "kernel": "split_kv"}
 
 
 def fdc_launch_count() -> int:
