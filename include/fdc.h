@@ -65,7 +65,9 @@ enum {
     FDC_DEV_ROW_RANGE     = 1,  /* fdc_kv_append: kv_row outside [0, rows): row skipped      */
     FDC_DEV_FRONTIER_WIDE = 2,  /* fdc_frontier: more ready fields than max_active: clamped, */
                                 /* the others wait for a later pass                          */
-    FDC_DEV_LEN_RANGE     = 4   /* fdc_state_init: a length outside [n_fixed+1, C]: clamped  */
+    FDC_DEV_LEN_RANGE     = 4,  /* fdc_state_init: a length outside [n_fixed+1, C]: clamped  */
+    FDC_DEV_TIMEOUT       = 8   /* fdc_decode_attn: a bounded in-kernel wait ran out; the    */
+                                /* launch's output is invalid                                */
 };
 
 typedef struct fdc_plan fdc_plan;
@@ -192,8 +194,8 @@ int fdc_decode_attn(const fdc_plan* plan, const fdc_kv_desc* kv, int32_t layer, 
  * `stream`.  *host_bits receives the FDC_DEV_* bits; returns FDC_ERR_DEVICE if non-zero. */
 int fdc_status(const fdc_plan* plan, int32_t* host_bits, int32_t clear, void* stream);
 
-/* Selects the attention kernel: 0 = automatic, 1 = CUDA-core reference kernel (any dtype),
- * other values as listed by fdc_kernel_name.  Unsupported combinations fall back to 1. */
+/* Selects the split-pass kernel: 0 = automatic (2 for bf16, 1 for fp32), 1 = CUDA-core kernel
+ * (any dtype), 2 = TMA + tensor-core MMA kernel (bf16).  Unsupported combinations use 1. */
 int fdc_set_attn_kernel(fdc_plan* plan, int32_t which);
 const char* fdc_kernel_name(int32_t which);
 

@@ -91,7 +91,7 @@ int fdc_attn_workspace_bytes(const fdc_plan* p, const fdc_kv_desc* kv, size_t* b
 int fdc_set_attn_kernel(fdc_plan* p, int32_t which)
 {
     if (!p) return FDC_ERR_NULL;
-    if (which < 0 || which > 1) return FDC_ERR_RANGE;
+    if (which < 0 || which > 2) return FDC_ERR_RANGE;
     p->attn_kernel = which;
     return FDC_OK;
 }
@@ -101,6 +101,7 @@ const char* fdc_kernel_name(int32_t which)
     switch (which) {
         case 0: return "auto";
         case 1: return "ref_cuda_core";
+        case 2: return "tma_mma_bf16";
         default: return nullptr;
     }
 }
@@ -144,6 +145,7 @@ int fdc_decode_attn(const fdc_plan* p, const fdc_kv_desc* kv, int32_t layer, con
     a.ws_o = (float*)d_workspace;
     a.ws_ml = a.ws_o + slots * a.mmax * kv->head_dim;
     a.n_cta = p->sm_count;
+    a.status = p->d_status;
 
     cudaStream_t st = (cudaStream_t)stream;
     Prof* pr = p->prof_on ? (Prof*)p->prof : nullptr;
@@ -156,7 +158,9 @@ int fdc_decode_attn(const fdc_plan* p, const fdc_kv_desc* kv, int32_t layer, con
         if (!e0 || !e1 || !e2) return set_cuda_error(cudaErrorMemoryAllocation);
         cudaEventRecord(e0, st);
     }
-    rc = launch_attn_ref(a, kv->dtype, kv->head_dim, st);
+    rc = FDC_ERR_SHAPE;
+    if (kv->dtype == FDC_BF16 && p->attn_kernel != 1) rc = launch_attn_mma(a, kv->head_dim, st);
+    if (rc == FDC_ERR_SHAPE) rc = launch_attn_ref(a, kv->dtype, kv->head_dim, st);
     if (rc) return rc;
     if (pr) cudaEventRecord(e1, st);
     rc = launch_attn_combine(a, kv->dtype, kv->head_dim, st);

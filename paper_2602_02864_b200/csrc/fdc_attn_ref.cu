@@ -263,13 +263,13 @@ int launch_ref_t(const AttnParams& p, cudaStream_t st)
 {
     size_t smem = sizeof(float) * ((size_t)64 * (D + 1) + 64 * D + 2 * (size_t)p.mmax * D + kWarps * 64 + 2 * p.mmax) +
                   sizeof(int) * (p.batch + 1);
-    static bool attr_set = false;
-    if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(attn_ref_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
-        if (e != cudaSuccess) return set_cuda_error(e);
-        attr_set = true;
-    }
     if (smem > 227 * 1024) return FDC_ERR_SHAPE;
+    static size_t attr_smem = 0;
+    if (smem > attr_smem) {
+        cudaError_t e = cudaFuncSetAttribute(attn_ref_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return set_cuda_error(e);
+        attr_smem = smem;
+    }
     attn_ref_kernel<T, D><<<p.n_cta, kThreads, smem, st>>>(p);
     note_launch();
     cudaError_t e = cudaGetLastError();

@@ -66,6 +66,7 @@ struct AttnParams {
     float*          ws_ml;           // [slots][mmax][2]
     int32_t         batch, hkv, hq, group, max_active, mmax, W, P, rows, ntile_max, n_cta;
     float           scale_log2;      // softmax scale * log2(e)
+    int32_t*        status;          // sticky FDC_DEV_* bits
 };
 
 extern int64_t g_launches;
@@ -73,6 +74,7 @@ void note_launch();
 int  set_cuda_error(cudaError_t e);                  // records the message, returns FDC_ERR_CUDA
 
 int launch_attn_ref(const AttnParams& p, int dtype, int head_dim, cudaStream_t st);
+int launch_attn_mma(const AttnParams& p, int head_dim, cudaStream_t st);
 int launch_attn_combine(const AttnParams& p, int dtype, int head_dim, cudaStream_t st);
 void prof_destroy(fdc_plan* plan);
 int  check_kv_desc(const fdc_plan* plan, const fdc_kv_desc* kv, int32_t layer);

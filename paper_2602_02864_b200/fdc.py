@@ -25,7 +25,7 @@ FDC_OK = 0
 FDC_ERR_NULL, FDC_ERR_CYCLE, FDC_ERR_RANGE, FDC_ERR_SHAPE = -1, -2, -3, -4
 FDC_ERR_DTYPE, FDC_ERR_WORKSPACE, FDC_ERR_CUDA, FDC_ERR_DEVICE = -5, -6, -7, -8
 FDC_F32, FDC_BF16 = 0, 1
-FDC_DEV_ROW_RANGE, FDC_DEV_FRONTIER_WIDE, FDC_DEV_LEN_RANGE = 1, 2, 4
+FDC_DEV_ROW_RANGE, FDC_DEV_FRONTIER_WIDE, FDC_DEV_LEN_RANGE, FDC_DEV_TIMEOUT = 1, 2, 4, 8
 
 c_i32, c_i64, c_vp, c_sz = ctypes.c_int32, ctypes.c_int64, ctypes.c_void_p, ctypes.c_size_t
 
