@@ -37,9 +37,15 @@ def log(*a):
     print(*a, file=sys.stderr, flush=True)
 
 
+LAYERS_OVERRIDE = None      # --layers: fewer layers of the same configuration (profiling captures)
+
+
 def get_workload(name: str):
     from paper_2602_02864_b200 import workloads as wl
-    return {"cfg0": wl.cfg0_tiny, "cfg1": wl.cfg1_7b, "cfg2": wl.cfg2_batched, "cfg3": wl.cfg3_wide}[name]()
+    if name == "cfg0":
+        return wl.cfg0_tiny()
+    f = {"cfg1": wl.cfg1_7b, "cfg2": wl.cfg2_batched, "cfg3": wl.cfg3_wide}[name]
+    return f() if LAYERS_OVERRIDE is None else f(layers=LAYERS_OVERRIDE)
 
 
 WORKLOAD_TEXT = {
@@ -400,7 +406,11 @@ def main():
     ap.add_argument("--impl", default="fdc", choices=["fdc", "reference"])
     ap.add_argument("--no-also", action="store_true", help="skip the short runs of the other configurations")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU baseline leg")
+    ap.add_argument("--layers", type=int, default=None,
+                    help="run only this many layers of the configuration (small ncu captures; not a bench number)")
     args = ap.parse_args()
+    global LAYERS_OVERRIDE
+    LAYERS_OVERRIDE = args.layers
     rank = int(os.environ.get("RANK", 0))
     world = int(os.environ.get("WORLD_SIZE", 1))
     if args.impl == "reference":

@@ -194,8 +194,9 @@ int fdc_decode_attn(const fdc_plan* plan, const fdc_kv_desc* kv, int32_t layer, 
  * `stream`.  *host_bits receives the FDC_DEV_* bits; returns FDC_ERR_DEVICE if non-zero. */
 int fdc_status(const fdc_plan* plan, int32_t* host_bits, int32_t clear, void* stream);
 
-/* Selects the split-pass kernel: 0 = automatic (2 for bf16, 1 for fp32), 1 = CUDA-core kernel
- * (any dtype), 2 = TMA + tensor-core MMA kernel (bf16).  Unsupported combinations use 1. */
+/* Selects the split-pass kernel: 0 = automatic (3 for bf16, 1 for fp32), 1 = CUDA-core kernel
+ * (any dtype), 2 = TMA + mma.sync kernel (bf16), 3 = TMA + tcgen05/TMEM kernel (bf16).
+ * Unsupported combinations use 1. */
 int fdc_set_attn_kernel(fdc_plan* plan, int32_t which);
 const char* fdc_kernel_name(int32_t which);
 

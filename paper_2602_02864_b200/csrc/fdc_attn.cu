@@ -91,7 +91,7 @@ int fdc_attn_workspace_bytes(const fdc_plan* p, const fdc_kv_desc* kv, size_t* b
 int fdc_set_attn_kernel(fdc_plan* p, int32_t which)
 {
     if (!p) return FDC_ERR_NULL;
-    if (which < 0 || which > 2) return FDC_ERR_RANGE;
+    if (which < 0 || which > 3) return FDC_ERR_RANGE;
     p->attn_kernel = which;
     return FDC_OK;
 }
@@ -102,6 +102,7 @@ const char* fdc_kernel_name(int32_t which)
         case 0: return "auto";
         case 1: return "ref_cuda_core";
         case 2: return "tma_mma_bf16";
+        case 3: return "tma_tcgen05_bf16";
         default: return nullptr;
     }
 }
@@ -159,7 +160,8 @@ int fdc_decode_attn(const fdc_plan* p, const fdc_kv_desc* kv, int32_t layer, con
         cudaEventRecord(e0, st);
     }
     rc = FDC_ERR_SHAPE;
-    if (kv->dtype == FDC_BF16 && p->attn_kernel != 1) rc = launch_attn_mma(a, kv->head_dim, st);
+    if (kv->dtype == FDC_BF16 && (p->attn_kernel == 0 || p->attn_kernel == 3)) rc = launch_attn_tc(a, kv->head_dim, st);
+    if (kv->dtype == FDC_BF16 && p->attn_kernel == 2) rc = launch_attn_mma(a, kv->head_dim, st);
     if (rc == FDC_ERR_SHAPE) rc = launch_attn_ref(a, kv->dtype, kv->head_dim, st);
     if (rc) return rc;
     if (pr) cudaEventRecord(e1, st);

@@ -2,11 +2,12 @@
 //
 // Sec. 3.3: all queries decoded in one forward pass (one per parallel field, times the GQA
 // heads of a KV head) share ONE read of the scene's KV rows.  Here a persistent CTA per SM
-// streams its share of the visited 64-row KV tiles through a ring of TMA-filled,
-// 128B-swizzled shared-memory stages; 8 consumer warps hold the query rows as MMA A
-// fragments (16-row blocks) and run an online softmax (running max / sum, fp32) per row.
-// Warps beyond the number of 16-row query blocks split each tile's rows between them
-// ("KV lanes") and merge at the end of a segment.  The per-branch row bitmaps (Eq. 1) are
+// streams its share of the visited 64-row KV tiles, as 32-row half tiles, through a ring of
+// TMA-filled, 128B-swizzled shared-memory stages; 8 consumer warps hold the query rows as MMA
+// A fragments (16-row blocks) and run an online softmax (running max / sum, fp32) per row.
+// When there are fewer 16-row query blocks than warps, the warps form several "KV lanes":
+// lane k takes every k-th stage for itself (whole stage: long independent MMA chains), and
+// the lanes' partial results are merged at the end of a segment.  The per-branch row bitmaps (Eq. 1) are
 // applied by select on the scores; tiles wholly inside the prefix skip masking.
 #include <cuda.h>
 #include <cuda_bf16.h>
@@ -15,7 +16,7 @@
 #include <mutex>
 #include <vector>
 
-#include "fdc_internal.h"
+#include "fdc_attn_common.cuh"
 
 using namespace fdc;
 
@@ -24,55 +25,9 @@ namespace {
 constexpr int NW = 8;                    // consumer warps
 constexpr int THREADS = (NW + 1) * 32;   // + 1 producer warp
 constexpr int TILE = FDC_TILE_ROWS;
-constexpr uint32_t SPIN_LIMIT = 1u << 22;
+constexpr int SROWS = 32;                // KV rows per shared-memory stage (half a tile)
+constexpr int HALVES = TILE / SROWS;     // stages per tile
 
-// ---------------------------------------------------------------- PTX wrappers
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
-{
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
-{
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar)
-{
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity)
-{
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(bar), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
-// Bounded wait: gives up after SPIN_LIMIT polls (or when another thread of the CTA gave up),
-// records FDC_DEV_TIMEOUT and returns false; the caller then skips all further work.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status)
-{
-    for (uint32_t i = 0; i < SPIN_LIMIT; ++i) {
-        if (mbar_try(bar, parity)) return true;
-        if ((i & 255u) == 255u) {
-            if (*abort_flag) return false;
-            __nanosleep(64);
-        }
-    }
-    *abort_flag = 1;
-    atomicOr(status, 8 /* FDC_DEV_TIMEOUT */);
-    return false;
-}
-__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int c0, int c1, int c2, int c3)
-{
-    asm volatile(
-        "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
-        ::"r"(dst), "l"(tm), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
-        : "memory");
-}
 __device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3)
 {
     asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
@@ -96,82 +51,36 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t*>(&v);
 }
-__device__ __forceinline__ float fast_exp2(float x)
-{
-    float y;
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-    return y;
-}
 __device__ __forceinline__ void consumer_bar() { asm volatile("bar.sync 1, %0;" ::"n"(NW * 32) : "memory"); }
 
 // Byte offset of the 16-byte chunk `dc` (0 .. D/8-1) of row `r` inside a K or V tile staged by
-// TMA with 128-byte swizzle: the tile is stored as D/64 panels of [64 rows][128 bytes]; inside
-// a panel the chunk index is XORed with (row mod 8).
+// TMA with 128-byte swizzle: the stage holds D/64 panels of [SROWS rows][128 bytes]; inside a
+// panel the chunk index is XORed with (row mod 8).
 __device__ __forceinline__ uint32_t tile_off(int r, int dc)
 {
-    return (uint32_t)((dc >> 3) * (TILE * 128) + r * 128 + (((dc & 7) ^ (r & 7)) << 4));
+    return (uint32_t)((dc >> 3) * (SROWS * 128) + r * 128 + (((dc & 7) ^ (r & 7)) << 4));
 }
 
-__device__ int scan_ntiles(const int32_t* __restrict__ ntiles, int batch, int* pre)
+// One staged half tile (SROWS rows) for one consumer warp.
+template <int D>
+__device__ __forceinline__ void process_stage(const uint32_t kbase, const uint32_t vbase, unsigned char* vgen,
+                                              const uint32_t (&qf)[D / 16][4], float (&o)[D / 8][4], float& m_lo, float& m_hi,
+                                              float& l_lo, float& l_hi, const bool masked, const uint64_t mk_lo,
+                                              const uint64_t mk_hi, const uint64_t zero_rows, const float c, const int lane)
 {
-    if (threadIdx.x < 32) {
-        int carry = 0;
-        for (int b0 = 0; b0 < batch; b0 += 32) {
-            int i = b0 + threadIdx.x;
-            int x = i < batch ? ntiles[i] : 0;
-            int inc = x;
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                int y = __shfl_up_sync(0xffffffffu, inc, o);
-                if ((int)threadIdx.x >= o) inc += y;
-            }
-            if (i < batch) pre[i] = carry + inc - x;
-            carry += __shfl_sync(0xffffffffu, inc, 31);
-        }
-        if (threadIdx.x == 0) pre[batch] = carry;
-    }
-    __syncthreads();
-    return pre[batch];
-}
-
-struct Segment {
-    int s, g, j0, j1, nt;
-    long long next_u;
-};
-// The run of units starting at u that belongs to one (scene, KV head) pair, cut at `hi`.
-__device__ __forceinline__ Segment decode_segment(long long u, long long hi, const int* pre, int hkv, int& s)
-{
-    while ((long long)pre[s + 1] * hkv <= u) ++s;
-    Segment sg;
-    sg.s = s;
-    sg.nt = pre[s + 1] - pre[s];
-    const long long u_scene = (long long)pre[s] * hkv;
-    sg.g = (int)((u - u_scene) / sg.nt);
-    const long long pair0 = u_scene + (long long)sg.g * sg.nt;
-    sg.j0 = (int)(u - pair0);
-    const long long end = pair0 + sg.nt < hi ? pair0 + sg.nt : hi;
-    sg.j1 = (int)(end - pair0);
-    sg.next_u = end;
-    return sg;
-}
-
-// One staged tile for one consumer warp: RW = rows of the tile this warp handles.
-template <int D, int RW>
-__device__ __forceinline__ void process_tile(const uint32_t kbase, const uint32_t vbase, unsigned char* vgen, const int ro,
-                                             const uint32_t (&qf)[D / 16][4], float (&o)[D / 8][4], float& m_lo, float& m_hi,
-                                             float& l_lo, float& l_hi, const bool masked, const uint64_t mk_lo,
-                                             const uint64_t mk_hi, const uint64_t zero_rows, const float c, const int lane)
-{
-    constexpr int NT = RW / 8;
+    constexpr int NT = SROWS / 8;
     float sacc[NT][4];
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) sacc[nt][0] = sacc[nt][1] = sacc[nt][2] = sacc[nt][3] = 0.f;
-    // S = Q K^T
+#if defined(FDC_EXP) && FDC_EXP == 1
+    return;
+#endif
+    // S = Q K^T: NT independent accumulator chains
 #pragma unroll
-    for (int nt = 0; nt < NT; ++nt) {
-        const int r = ro + nt * 8 + (lane & 7);
+    for (int ks = 0; ks < D / 16; ks += 2) {
 #pragma unroll
-        for (int ks = 0; ks < D / 16; ks += 2) {
+        for (int nt = 0; nt < NT; ++nt) {
+            const int r = nt * 8 + (lane & 7);
             uint32_t b0, b1, b2, b3;
             ldsm_x4(kbase + tile_off(r, 2 * ks + (lane >> 3)), b0, b1, b2, b3);
             mma_bf16(sacc[nt], qf[ks], b0, b1);
@@ -182,7 +91,7 @@ __device__ __forceinline__ void process_tile(const uint32_t kbase, const uint32_
         // rows nobody may see can hold anything: clear their V so that 0 * NaN cannot arise
         uint64_t z = zero_rows;
         while (z) {
-            const int r = ro + __ffsll((long long)z) - 1;
+            const int r = __ffsll((long long)z) - 1;
             z &= z - 1;
             for (int i = lane; i < D / 4; i += 32)        // D*2 bytes = D/4 words of 8 bytes
                 *reinterpret_cast<uint2*>(vgen + tile_off(r, i >> 1) + (i & 1) * 8) = make_uint2(0u, 0u);
@@ -212,37 +121,44 @@ __device__ __forceinline__ void process_tile(const uint32_t kbase, const uint32_
     const float mn_lo = fmaxf(m_lo, mx_lo), mn_hi = fmaxf(m_hi, mx_hi);
     const float ms_lo = mn_lo == -INFINITY ? 0.f : mn_lo * c;      // a row that has seen nothing yet
     const float ms_hi = mn_hi == -INFINITY ? 0.f : mn_hi * c;
-    const float a_lo = fast_exp2(m_lo * c - ms_lo), a_hi = fast_exp2(m_hi * c - ms_hi);
-    m_lo = mn_lo;
-    m_hi = mn_hi;
-    float s_lo = 0.f, s_hi = 0.f;
+    // the running maxima settle after a few tiles: rescale only when one of them moved
+    const bool moved = (mn_lo != m_lo) || (mn_hi != m_hi);
+    if (__any_sync(0xffffffffu, moved)) {
+        const float a_lo = fast_exp2(m_lo * c - ms_lo), a_hi = fast_exp2(m_hi * c - ms_hi);
+        l_lo *= a_lo;
+        l_hi *= a_hi;
+#pragma unroll
+        for (int i = 0; i < D / 8; ++i) {
+            o[i][0] *= a_lo;
+            o[i][1] *= a_lo;
+            o[i][2] *= a_hi;
+            o[i][3] *= a_hi;
+        }
+        m_lo = mn_lo;
+        m_hi = mn_hi;
+    }
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) {
         sacc[nt][0] = fast_exp2(fmaf(sacc[nt][0], c, -ms_lo));
         sacc[nt][1] = fast_exp2(fmaf(sacc[nt][1], c, -ms_lo));
         sacc[nt][2] = fast_exp2(fmaf(sacc[nt][2], c, -ms_hi));
         sacc[nt][3] = fast_exp2(fmaf(sacc[nt][3], c, -ms_hi));
-        s_lo += sacc[nt][0] + sacc[nt][1];
-        s_hi += sacc[nt][2] + sacc[nt][3];
+        l_lo += sacc[nt][0] + sacc[nt][1];
+        l_hi += sacc[nt][2] + sacc[nt][3];
     }
-    l_lo = fmaf(l_lo, a_lo, s_lo);
-    l_hi = fmaf(l_hi, a_hi, s_hi);
-#pragma unroll
-    for (int i = 0; i < D / 8; ++i) {
-        o[i][0] *= a_lo;
-        o[i][1] *= a_lo;
-        o[i][2] *= a_hi;
-        o[i][3] *= a_hi;
-    }
+#if defined(FDC_EXP) && FDC_EXP == 2
+    o[0][0] += sacc[0][0] + sacc[1][1] + sacc[2][2] + sacc[3][3];
+    return;
+#endif
     // O += P V
 #pragma unroll
-    for (int kk = 0; kk < RW / 16; ++kk) {
+    for (int kk = 0; kk < SROWS / 16; ++kk) {
         uint32_t pa[4];
         pa[0] = pack_bf16(sacc[2 * kk][0], sacc[2 * kk][1]);
         pa[1] = pack_bf16(sacc[2 * kk][2], sacc[2 * kk][3]);
         pa[2] = pack_bf16(sacc[2 * kk + 1][0], sacc[2 * kk + 1][1]);
         pa[3] = pack_bf16(sacc[2 * kk + 1][2], sacc[2 * kk + 1][3]);
-        const int r = ro + kk * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
+        const int r = kk * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
 #pragma unroll
         for (int np = 0; np < D / 16; ++np) {
             uint32_t b0, b1, b2, b3;
@@ -258,7 +174,7 @@ __global__ void __launch_bounds__(THREADS, 1)
 attn_mma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
                 const int nstage)
 {
-    constexpr int STAGE_BYTES = 2 * TILE * D * 2;          // K tile + V tile
+    constexpr int STAGE_BYTES = 2 * SROWS * D * 2;         // K rows + V rows of half a tile
     constexpr int MERGE_WARP_FLOATS = (D / 8 * 4 + 4) * 32;
     extern __shared__ unsigned char smem_dyn[];
     unsigned char* smem = reinterpret_cast<unsigned char*>(((uintptr_t)smem_dyn + 1023) & ~(uintptr_t)1023);
@@ -289,36 +205,46 @@ attn_mma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, co
     volatile int* abortp = &abort_flag;
 
     if (warp == NW) {
-        // ------------------------------------------------ producer: one thread feeds the ring
-        if (lane == 0) {
-            int s = 0;
-            uint32_t it = 0;
-            long long u = lo;
-            bool ok = true;
-            while (u < hi && ok) {
-                const Segment sg = decode_segment(u, hi, pre, p.hkv, s);
-                for (int j = sg.j0; j < sg.j1; ++j, ++it) {
-                    const int st = it % nstage;
-                    const uint32_t ph = (it / nstage) & 1;
-                    if (!mbar_wait(empty0 + 8 * st, ph ^ 1, abortp, p.status)) { ok = false; break; }
-                    const int tile = p.tiles[(size_t)sg.s * p.ntile_max + j];
-                    const uint32_t dst = smem_u32(stages + (size_t)st * STAGE_BYTES);
-                    mbar_expect_tx(full0 + 8 * st, STAGE_BYTES);
+        // ------------------------------------------------ producer warp: lane 0 feeds the ring; the
+        // tile ids are fetched 32 at a time by the whole warp so that no global-load latency sits
+        // between two TMA issues
+        int s = 0;
+        uint32_t it = 0;
+        long long u = lo;
+        int ok = 1;
+        while (u < hi && ok) {
+            const Segment sg = decode_segment(u, hi, pre, p.hkv, s);
+            for (int jb = sg.j0; jb < sg.j1 && ok; jb += 32) {
+                const int jn = sg.j1 - jb < 32 ? sg.j1 - jb : 32;
+                const int my_tile = lane < jn ? p.tiles[(size_t)sg.s * p.ntile_max + jb + lane] : 0;
+                for (int k = 0; k < jn && ok; ++k) {
+                    const int tile = __shfl_sync(0xffffffffu, my_tile, k);
+                    if (lane == 0) {
+                        for (int half = 0; half < HALVES && ok; ++half, ++it) {
+                            const int st = it % nstage;
+                            const uint32_t ph = (it / nstage) & 1;
+                            if (!mbar_wait(empty0 + 8 * st, ph ^ 1, abortp, p.status)) { ok = 0; break; }
+                            const int row0 = tile * TILE + half * SROWS;
+                            const uint32_t dst = smem_u32(stages + (size_t)st * STAGE_BYTES);
+                            mbar_expect_tx(full0 + 8 * st, STAGE_BYTES);
 #pragma unroll
-                    for (int h = 0; h < D / 64; ++h) {
-                        tma_load_4d(dst + h * (TILE * 128), &tm_k, full0 + 8 * st, h * 64, tile * TILE, sg.g, sg.s);
-                        tma_load_4d(dst + TILE * D * 2 + h * (TILE * 128), &tm_v, full0 + 8 * st, h * 64, tile * TILE, sg.g, sg.s);
+                            for (int h = 0; h < D / 64; ++h) {
+                                tma_load_4d(dst + h * (SROWS * 128), &tm_k, full0 + 8 * st, h * 64, row0, sg.g, sg.s);
+                                tma_load_4d(dst + SROWS * D * 2 + h * (SROWS * 128), &tm_v, full0 + 8 * st, h * 64, row0, sg.g, sg.s);
+                            }
+                        }
                     }
+                    ok = __shfl_sync(0xffffffffu, ok, 0);
                 }
-                u = sg.next_u;
             }
-            if (!ok) {
-                // give the copies already in flight a bounded chance to land before the CTA ends
-                const uint32_t first = it > (uint32_t)nstage ? it - nstage : 0;
-                for (uint32_t k = first; k < it; ++k) {
-                    const uint32_t bar = full0 + 8 * (k % nstage), ph = (k / nstage) & 1;
-                    for (uint32_t i = 0; i < (1u << 16) && !mbar_try(bar, ph); ++i) __nanosleep(64);
-                }
+            u = sg.next_u;
+        }
+        if (!ok && lane == 0) {
+            // give the copies already in flight a bounded chance to land before the CTA ends
+            const uint32_t first = it > (uint32_t)nstage ? it - nstage : 0;
+            for (uint32_t k = first; k < it; ++k) {
+                const uint32_t bar = full0 + 8 * (k % nstage), ph = (k / nstage) & 1;
+                for (uint32_t i = 0; i < (1u << 16) && !mbar_try(bar, ph); ++i) __nanosleep(64);
             }
         }
         return;
@@ -340,7 +266,6 @@ attn_mma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, co
         const int kvl = nmb == 1 ? 4 : (nmb == 2 ? 4 : (nmb <= 4 ? 2 : 1));
         const bool active = warp < nmb * kvl;
         const int mb = active ? warp % nmb : 0, kl = active ? warp / nmb : 0;
-        const int rw = TILE / kvl, ro = kl * rw;
         const int row_lo = mb * 16 + gq, row_hi = row_lo + 8;
         const int b_lo = row_lo / p.group, b_hi = row_hi / p.group;
 
@@ -368,39 +293,49 @@ attn_mma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, co
         const uint64_t* mrow_lo = p.mask + ((size_t)sg.s * p.max_active + (row_lo < M ? b_lo : 0)) * p.W;
         const uint64_t* mrow_hi = p.mask + ((size_t)sg.s * p.max_active + (row_hi < M ? b_hi : 0)) * p.W;
 
-        for (int j = sg.j0; j < sg.j1; ++j, ++it) {
+        for (int jb = sg.j0; jb < sg.j1; jb += 32) {
+          const int jn = sg.j1 - jb < 32 ? sg.j1 - jb : 32;
+          const int my_tile = lane < jn ? p.tiles[(size_t)sg.s * p.ntile_max + jb + lane] : 0;
+          for (int q = HALVES * jb; q < HALVES * (jb + jn); ++q, ++it) {
+            const int tile = __shfl_sync(0xffffffffu, my_tile, q / HALVES - jb);
             const int st = it % nstage;
             const uint32_t ph = (it / nstage) & 1;
-            if (alive && !mbar_wait(full0 + 8 * st, ph, abortp, p.status)) alive = false;
-            if (alive && active) {
-                const int tile = p.tiles[(size_t)sg.s * p.ntile_max + j];
+            const bool mine = active && ((q - HALVES * sg.j0) % kvl) == kl;     // this KV lane's stage
+            if (alive) {
+                // every warp follows the ring (its arrival is counted), only the owners read the stage
+                if (mine) {
+                    if (!mbar_wait(full0 + 8 * st, ph, abortp, p.status)) alive = false;
+                } else {
+                    int ok = 1;
+                    if (lane == 0) ok = mbar_wait(full0 + 8 * st, ph, abortp, p.status);
+                    if (!__shfl_sync(0xffffffffu, ok, 0)) alive = false;
+                }
+            }
+            if (alive && mine) {
                 const int r0 = tile * TILE;
-                const bool masked = r0 + TILE > p.P;
+                const int sh = (q % HALVES) * SROWS;
+                const bool masked = r0 + sh + SROWS > p.P;
+                const uint64_t stage_bits = SROWS == 64 ? ~0ull : ((1ull << (SROWS & 63)) - 1ull);
                 uint64_t mk_lo = ~0ull, mk_hi = ~0ull, zero_rows = 0ull;
                 if (masked) {
-                    mk_lo = row_lo < M ? tile_rowmask(mrow_lo, p.W, p.P, tile) >> ro : 0ull;
-                    mk_hi = row_hi < M ? tile_rowmask(mrow_hi, p.W, p.P, tile) >> ro : 0ull;
+                    mk_lo = row_lo < M ? (tile_rowmask(mrow_lo, p.W, p.P, tile) >> sh) & stage_bits : 0ull;
+                    mk_hi = row_hi < M ? (tile_rowmask(mrow_hi, p.W, p.P, tile) >> sh) & stage_bits : 0ull;
                     uint64_t um = 0ull;                      // rows of the tile visible to any branch
                     for (int b = lane; b < A; b += 32)
                         um |= tile_rowmask(p.mask + ((size_t)sg.s * p.max_active + b) * p.W, p.W, p.P, tile);
                     const uint32_t ul = __reduce_or_sync(0xffffffffu, (uint32_t)um);
                     const uint32_t uh = __reduce_or_sync(0xffffffffu, (uint32_t)(um >> 32));
-                    um = ((uint64_t)uh << 32) | ul;
-                    zero_rows = (~um >> ro) & (rw == 64 ? ~0ull : ((1ull << rw) - 1ull));
+                    zero_rows = (~((((uint64_t)uh << 32) | ul) >> sh)) & stage_bits;
                 }
                 unsigned char* stg = stages + (size_t)st * STAGE_BYTES;
-                const uint32_t kb = smem_u32(stg), vb = kb + TILE * D * 2;
-                unsigned char* vgen = stg + TILE * D * 2;
-                if (kvl == 4)
-                    process_tile<D, 16>(kb, vb, vgen, ro, qf, o, m_lo, m_hi, l_lo, l_hi, masked, mk_lo, mk_hi, zero_rows, c, lane);
-                else if (kvl == 2)
-                    process_tile<D, 32>(kb, vb, vgen, ro, qf, o, m_lo, m_hi, l_lo, l_hi, masked, mk_lo, mk_hi, zero_rows, c, lane);
-                else
-                    process_tile<D, 64>(kb, vb, vgen, ro, qf, o, m_lo, m_hi, l_lo, l_hi, masked, mk_lo, mk_hi, zero_rows, c, lane);
+                const uint32_t kb = smem_u32(stg), vb = kb + SROWS * D * 2;
+                process_stage<D>(kb, vb, stg + SROWS * D * 2, qf, o, m_lo, m_hi, l_lo, l_hi, masked, mk_lo, mk_hi, zero_rows,
+                                 c, lane);
                 if (masked) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(empty0 + 8 * st);
+          }
         }
 
         // ---- end of segment: merge the KV lanes, write the partial (m, l, O)
@@ -493,10 +428,10 @@ PFN_cuTensorMapEncodeTiled get_encode()
 struct MapKey {
     const void* base;
     int64_t ss, sh, sr;
-    int32_t batch, hkv, rows, d;
+    int32_t batch, hkv, rows, d, box_rows;
     bool operator==(const MapKey& o) const
     {
-        return base == o.base && ss == o.ss && sh == o.sh && sr == o.sr && batch == o.batch && hkv == o.hkv && rows == o.rows && d == o.d;
+        return base == o.base && ss == o.ss && sh == o.sh && sr == o.sr && batch == o.batch && hkv == o.hkv && rows == o.rows && d == o.d && box_rows == o.box_rows;
     }
 };
 struct MapCache {
@@ -505,9 +440,9 @@ struct MapCache {
 };
 MapCache g_maps;
 
-int get_map(const void* base, const AttnParams& p, int d, CUtensorMap* out)
+int get_map(const void* base, const AttnParams& p, int d, int box_rows, CUtensorMap* out)
 {
-    MapKey key{base, p.stride_scene, p.stride_head, p.stride_row, p.batch, p.hkv, p.rows, d};
+    MapKey key{base, p.stride_scene, p.stride_head, p.stride_row, p.batch, p.hkv, p.rows, d, box_rows};
     std::lock_guard<std::mutex> lk(g_maps.mu);
     for (auto& it : g_maps.items)
         if (it.first == key) {
@@ -520,7 +455,7 @@ int get_map(const void* base, const AttnParams& p, int d, CUtensorMap* out)
     // a dimension of extent 1 still needs a legal (multiple of 16 bytes, non-zero) stride
     auto str = [](int64_t s, int64_t fallback) { return (cuuint64_t)((s > 0 ? s : fallback) * 2); };
     cuuint64_t strides[3] = {str(p.stride_row, d), str(p.stride_head, (int64_t)d * p.rows), str(p.stride_scene, (int64_t)d * p.rows * p.hkv)};
-    cuuint32_t box[4] = {64, TILE, 1, 1};
+    cuuint32_t box[4] = {64, (cuuint32_t)box_rows, 1, 1};
     cuuint32_t estr[4] = {1, 1, 1, 1};
     alignas(64) CUtensorMap tm;
     CUresult r = enc(&tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
@@ -536,11 +471,11 @@ int get_map(const void* base, const AttnParams& p, int d, CUtensorMap* out)
 template <int D>
 int launch_t(const AttnParams& p, cudaStream_t st)
 {
-    constexpr int STAGE_BYTES = 2 * TILE * D * 2;
+    constexpr int STAGE_BYTES = 2 * SROWS * D * 2;
     constexpr int MERGE_BYTES = 6 * (D / 8 * 4 + 4) * 32 * 4;
-    const size_t fixed = 1024 + MERGE_BYTES + 2 * 8 * 8 + sizeof(int) * (p.batch + 1) + 64;
+    const size_t fixed = 1024 + MERGE_BYTES + 2 * 16 * 8 + sizeof(int) * (p.batch + 1) + 64;
     int nstage = (int)((227 * 1024 - 256 - fixed) / STAGE_BYTES);   // 256: static shared + slack
-    if (nstage > 8) nstage = 8;
+    if (nstage > 16) nstage = 16;
     if (nstage < 2) return FDC_ERR_SHAPE;
     const size_t smem = fixed + (size_t)nstage * STAGE_BYTES;
     static size_t attr_smem = 0;
@@ -550,9 +485,9 @@ int launch_t(const AttnParams& p, cudaStream_t st)
         attr_smem = smem;
     }
     alignas(64) CUtensorMap tk, tv;
-    int rc = get_map(p.k, p, D, &tk);
+    int rc = get_map(p.k, p, D, SROWS, &tk);
     if (rc) return rc;
-    rc = get_map(p.v, p, D, &tv);
+    rc = get_map(p.v, p, D, SROWS, &tv);
     if (rc) return rc;
     attn_mma_kernel<D><<<p.n_cta, THREADS, smem, st>>>(p, tk, tv, nstage);
     note_launch();
@@ -563,6 +498,11 @@ int launch_t(const AttnParams& p, cudaStream_t st)
 }  // namespace
 
 namespace fdc {
+
+int get_kv_tensor_map(const void* base, const AttnParams& p, int head_dim, int box_rows, void* out_map)
+{
+    return get_map(base, p, head_dim, box_rows, reinterpret_cast<CUtensorMap*>(out_map));
+}
 
 // bf16 only.  Returns FDC_ERR_SHAPE when the tensor map cannot describe the cache (the caller
 // then uses the CUDA-core kernel).

@@ -75,6 +75,7 @@ int  set_cuda_error(cudaError_t e);                  // records the message, ret
 
 int launch_attn_ref(const AttnParams& p, int dtype, int head_dim, cudaStream_t st);
 int launch_attn_mma(const AttnParams& p, int head_dim, cudaStream_t st);
+int launch_attn_tc(const AttnParams& p, int head_dim, cudaStream_t st);
 int launch_attn_combine(const AttnParams& p, int dtype, int head_dim, cudaStream_t st);
 void prof_destroy(fdc_plan* plan);
 int  check_kv_desc(const fdc_plan* plan, const fdc_kv_desc* kv, int32_t layer);

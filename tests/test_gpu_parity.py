@@ -24,10 +24,11 @@ def test_cfg0_tiny_every_step():
     assert r["steps"] == 48 and r["checked"] == 96 * 4
 
 
-@pytest.mark.parametrize("kernel", [1, 2])
+@pytest.mark.parametrize("kernel", [1, 2, 3])
 @pytest.mark.parametrize("head_dim", [64, 128])
-def test_cfg0_tiny_bf16_both_kernels(kernel, head_dim):
-    """The bf16 variant of the tiny case through the CUDA-core kernel (1) and the TMA + MMA kernel (2)."""
+def test_cfg0_tiny_bf16_all_kernels(kernel, head_dim):
+    """The bf16 variant of the tiny case through the CUDA-core kernel (1), the TMA + mma.sync
+    kernel (2) and the TMA + tcgen05 kernel (3)."""
     w = wl.cfg0_tiny()
     w.dtype, w.head_dim = "bf16", head_dim
     run_and_compare(w, kernel=kernel)
