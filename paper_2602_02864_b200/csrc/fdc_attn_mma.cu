@@ -72,9 +72,6 @@ __device__ __forceinline__ void process_stage(const uint32_t kbase, const uint32
     float sacc[NT][4];
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) sacc[nt][0] = sacc[nt][1] = sacc[nt][2] = sacc[nt][3] = 0.f;
-#if defined(FDC_EXP) && FDC_EXP == 1
-    return;
-#endif
     // S = Q K^T: NT independent accumulator chains
 #pragma unroll
     for (int ks = 0; ks < D / 16; ks += 2) {
@@ -146,10 +143,6 @@ __device__ __forceinline__ void process_stage(const uint32_t kbase, const uint32
         l_lo += sacc[nt][0] + sacc[nt][1];
         l_hi += sacc[nt][2] + sacc[nt][3];
     }
-#if defined(FDC_EXP) && FDC_EXP == 2
-    o[0][0] += sacc[0][0] + sacc[1][1] + sacc[2][2] + sacc[3][3];
-    return;
-#endif
     // O += P V
 #pragma unroll
     for (int kk = 0; kk < SROWS / 16; ++kk) {
