@@ -45,6 +45,7 @@ extern "C" {
 #define FDC_TILE_ROWS   64   /* KV rows per tile of the visited-tile list                   */
 #define FDC_MAX_QROWS   128  /* max_active * (hq / hkv): query rows served by one KV read   */
 #define FDC_MAX_BATCH   4096 /* scenes per call                                             */
+#define FDC_STATIC_WS_BYTES (16u << 20) /* built-in scratch of fdc_decode_attn_static, per GPU  */
 
 enum {
     FDC_OK            =  0,
@@ -55,7 +56,9 @@ enum {
     FDC_ERR_DTYPE     = -5,  /* dtype is neither FDC_F32 nor FDC_BF16                       */
     FDC_ERR_WORKSPACE = -6,  /* workspace missing, misaligned or smaller than required      */
     FDC_ERR_CUDA      = -7,  /* a CUDA runtime call failed (see fdc_last_cuda_error)        */
-    FDC_ERR_DEVICE    = -8   /* fdc_status: the device recorded an anomaly                  */
+    FDC_ERR_DEVICE    = -8,  /* fdc_status: the device recorded an anomaly                  */
+    FDC_ERR_STATIC_LIMIT = -9 /* fdc_decode_attn_static: the problem needs more scratch than */
+                             /* FDC_STATIC_WS_BYTES; nothing was launched                   */
 };
 
 enum { FDC_F32 = 0, FDC_BF16 = 1 };
@@ -189,6 +192,38 @@ int fdc_decode_attn(const fdc_plan* plan, const fdc_kv_desc* kv, int32_t layer, 
                     const uint64_t* d_mask, const int32_t* d_tiles, const int32_t* d_ntiles,
                     const void* d_q, void* d_out, float scale, void* d_workspace, size_t ws_bytes,
                     void* stream);
+
+/* fdc_decode_attn without a workspace argument, for callers that cannot allocate device
+ * memory.  (The paper has no counterpart: it describes no memory management at all; this is
+ * a deployment variant of the call above and computes exactly the same thing.)
+ *
+ * Meant for hosts that may not allocate once they run: an in-vehicle runtime whose device
+ * memory budget is fixed at start-up and whose decode loop must not call cudaMalloc (it
+ * synchronises the device, has no latency bound and fails once the KV pool owns the GPU), or
+ * a plugin-style host whose per-step call is forbidden to allocate.  The split partials go
+ * to a buffer inside the library image instead: FDC_STATIC_WS_BYTES (16 MiB) of device
+ * memory on every GPU that loads the library, held until the process exits.
+ *
+ *   - Limit: fdc_attn_workspace_bytes(plan, kv) must not exceed FDC_STATIC_WS_BYTES, else
+ *     FDC_ERR_STATIC_LIMIT is returned and nothing is launched.  The four bf16/fp32
+ *     configurations of up to 16 scenes x 8 KV heads with 64 query rows per KV head fit; 64
+ *     scenes x 128 query rows do not.
+ *   - The call itself makes no device allocation and frees nothing (no cudaMalloc / cudaFree,
+ *     no allocating library routine); inputs and outputs are still the caller's.  Keep
+ *     fdc_profile off: profiling creates CUDA events.
+ *   - The FIRST call on a device looks up the buffer's device address (a host-side query made
+ *     with that device current, checked, then remembered).  Make that first call during
+ *     start-up, before any stream capture is begun.  The CUDA device current at the call must
+ *     be the plan's device (FDC_ERR_RANGE otherwise).
+ *   - All calls on a GPU share the one buffer, and it keeps whatever the last call left.  No
+ *     part of it has to start at zero (each call's combine pass reads only partials that the
+ *     same call's split pass wrote), so it is never cleared.  Two calls whose kernels can
+ *     overlap on the GPU (different streams, or several host threads or plans on one device)
+ *     race on it and corrupt each other's results: issue them on one stream or order them
+ *     with events. */
+int fdc_decode_attn_static(const fdc_plan* plan, const fdc_kv_desc* kv, int32_t layer, const int32_t* d_n_active,
+                           const uint64_t* d_mask, const int32_t* d_tiles, const int32_t* d_ntiles,
+                           const void* d_q, void* d_out, float scale, void* stream);
 
 /* Reads (and with clear != 0 resets) the sticky device status word after synchronising
  * `stream`.  *host_bits receives the FDC_DEV_* bits; returns FDC_ERR_DEVICE if non-zero. */

@@ -49,6 +49,7 @@ const char* fdc_strerror(int code)
         case FDC_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
         case FDC_ERR_CUDA: return "CUDA runtime error";
         case FDC_ERR_DEVICE: return "device recorded an anomaly";
+        case FDC_ERR_STATIC_LIMIT: return "problem needs more scratch than the built-in static buffer (FDC_STATIC_WS_BYTES)";
         default: return "unknown error";
     }
 }

@@ -24,6 +24,8 @@ FDC_MAX_NODES, FDC_TILE_ROWS, FDC_MAX_QROWS, FDC_MAX_BATCH = 64, 64, 128, 4096
 FDC_OK = 0
 FDC_ERR_NULL, FDC_ERR_CYCLE, FDC_ERR_RANGE, FDC_ERR_SHAPE = -1, -2, -3, -4
 FDC_ERR_DTYPE, FDC_ERR_WORKSPACE, FDC_ERR_CUDA, FDC_ERR_DEVICE = -5, -6, -7, -8
+FDC_ERR_STATIC_LIMIT = -9
+FDC_STATIC_WS_BYTES = 16 << 20
 FDC_F32, FDC_BF16 = 0, 1
 FDC_DEV_ROW_RANGE, FDC_DEV_FRONTIER_WIDE, FDC_DEV_LEN_RANGE, FDC_DEV_TIMEOUT = 1, 2, 4, 8
 
@@ -66,6 +68,8 @@ _kv_append = _sig("fdc_kv_append", c_i32, c_vp, ctypes.POINTER(fdc_kv_desc), c_i
 _attn_ws = _sig("fdc_attn_workspace_bytes", c_i32, c_vp, ctypes.POINTER(fdc_kv_desc), ctypes.POINTER(c_sz))
 _decode_attn = _sig("fdc_decode_attn", c_i32, c_vp, ctypes.POINTER(fdc_kv_desc), c_i32, c_vp, c_vp, c_vp, c_vp,
                     c_vp, c_vp, ctypes.c_float, c_vp, c_sz, c_vp)
+_decode_attn_static = _sig("fdc_decode_attn_static", c_i32, c_vp, ctypes.POINTER(fdc_kv_desc), c_i32, c_vp, c_vp, c_vp,
+                           c_vp, c_vp, c_vp, ctypes.c_float, c_vp)
 _status = _sig("fdc_status", c_i32, c_vp, ctypes.POINTER(c_i32), c_i32, c_vp)
 _set_attn_kernel = _sig("fdc_set_attn_kernel", c_i32, c_vp, c_i32)
 _kernel_name = _sig("fdc_kernel_name", ctypes.c_char_p, c_i32)
@@ -184,6 +188,16 @@ def fdc_decode_attn(plan, kv: fdc_kv_desc, layer, d_n_active, d_mask, d_tiles, d
     _check(_decode_attn(plan, ctypes.byref(kv), layer, _ptr(d_n_active), _ptr(d_mask), _ptr(d_tiles), _ptr(d_ntiles),
                         _ptr(d_q), _ptr(d_out), float(scale), _ptr(d_workspace), int(ws_bytes), _stream(stream)),
            "fdc_decode_attn")
+
+
+def fdc_decode_attn_static(plan, kv: fdc_kv_desc, layer, d_n_active, d_mask, d_tiles, d_ntiles, d_q, d_out, scale,
+                           stream=None) -> None:
+    """fdc_decode_attn for callers that may not allocate device memory: the split partials go to
+    the library's built-in 16 MiB buffer (shared by all calls on the GPU; overlapping calls race).
+    Raises FdcError(FDC_ERR_STATIC_LIMIT) when the problem needs more scratch than that."""
+    _check(_decode_attn_static(plan, ctypes.byref(kv), layer, _ptr(d_n_active), _ptr(d_mask), _ptr(d_tiles),
+                               _ptr(d_ntiles), _ptr(d_q), _ptr(d_out), float(scale), _stream(stream)),
+           "fdc_decode_attn_static")
 
 
 def fdc_status(plan, clear: bool = False, stream=None) -> int:
