@@ -161,7 +161,8 @@ int fdc_decode_attn(const fdc_plan* p, const fdc_kv_desc* kv, int32_t layer, con
     }
     rc = FDC_ERR_SHAPE;
     if (kv->dtype == FDC_BF16 && (p->attn_kernel == 0 || p->attn_kernel == 3)) rc = launch_attn_tc(a, kv->head_dim, st);
-    if (kv->dtype == FDC_BF16 && p->attn_kernel == 2) rc = launch_attn_mma(a, kv->head_dim, st);
+    if (kv->dtype == FDC_BF16 && (p->attn_kernel == 2 || (rc == FDC_ERR_SHAPE && p->attn_kernel != 1)))
+        rc = launch_attn_mma(a, kv->head_dim, st);
     if (rc == FDC_ERR_SHAPE) rc = launch_attn_ref(a, kv->dtype, kv->head_dim, st);
     if (rc) return rc;
     if (pr) cudaEventRecord(e1, st);

@@ -1,25 +1,31 @@
-// Split-KV pass for bf16 caches on the 5th-generation tensor cores (tcgen05 + TMEM).
+// Split-KV pass for bf16 caches (head_dim 128) on the 5th-generation tensor cores (tcgen05 + TMEM).
 //
 // Sec. 3.3: the queries of all parallel fields of a scene, times the GQA heads of a KV head,
-// share ONE read of the KV rows.  Here they form the (zero-padded) 128-row M side of two
-// tcgen05 MMAs per 64-row KV tile: S = Q K^T (accumulator in TMEM, 64 columns, double
-// buffered) and O += P V (accumulator in TMEM, head_dim columns).  One persistent CTA per SM:
-//   warps 8, 10 TMA producers: K tiles and V tiles into two 128B-swizzled shared-memory rings
-//               (a K stage is free again after its S = Q K^T, a V stage after its O += P V)
-//   warp 9      MMA issuer (one elected thread), allocates / frees TMEM; S = Q K^T is issued up
-//               to four tiles ahead of the softmax (four score buffers in TMEM)
-//   warps 0-7   softmax.  A warp can only read the 32 TMEM lanes of its quadrant (warp % 4), so
-//               when there are at most 32 (64) query rows they are replicated 4 (2) times along
-//               M: every quadrant then holds a copy of each score row and the 8 warps split the
-//               64 score columns of a row between them (8, 16 or 32 columns per thread).  Each
-//               thread applies its branch's row bitmap (Eq. 1) by select, exponentiates against
-//               the row's reference maximum and writes its slice of P (bf16) to shared memory,
-//               the A operand of P V.
-// The reference maximum of a row is shared by its threads and only raised when some slice
-// maximum exceeds it by more than 2^8 (found with one barrier-wide OR per tile); the slices'
-// maxima are then exchanged through shared memory and the accumulator row is rescaled in
-// TMEM.  Results are exact either way: sum and accumulator use the same reference.
+// share ONE read of the KV rows.  The kernel is written in the transposed form, with the KV
+// rows on the M side of the MMAs and the (few) query rows on the N side, so that the tensor
+// work scales with the real number of queries and every TMEM lane / softmax thread owns a
+// real KV row:
+//     S^T = K Q^T      M = 128 KV rows (one "round" = two 64-row tiles of the visited-tile
+//                      list), N = NP query rows (16/32/64/128), K = head_dim;  A = the K tiles
+//                      as TMA left them in shared memory, B = Q^T staged once per segment
+//     O^T += V^T P^T   M = head_dim, N = NP, K = 128 KV rows;  A = the V tiles (M-major), B =
+//                      P^T written by the softmax threads (N-major), accumulator in TMEM
+// One persistent CTA per SM:
+//   warps 8, 10  TMA producers: K stages and V stages (128 rows, 128B swizzle) of two rings
+//   warp 9       MMA issuer (one elected thread); allocates / frees TMEM.  S^T is double
+//                buffered in TMEM, so K Q^T of round r+1 overlaps the softmax of round r
+//   warp 11      clears the V rows that no branch may see (they can hold anything, NaN included,
+//                and 0 * NaN must not reach the accumulator) and then releases the stage to the MMA
+//   warps 0-7    softmax.  Thread = one KV row of the round (TMEM lane) x half of the query
+//                columns.  Eq. 1 is applied by select from the branches' row bitmaps; prefix
+//                tiles skip it.
+// The softmax reference of a query column is raised lazily: it is set from the column maximum
+// of the first round and raised again only when some score exceeds it by more than 2^8 (one
+// barrier-wide OR per round detects that).  Sum and accumulator use the same reference, so the
+// result is exact; the column sums are kept per thread and reduced at the end of a segment.
 #include <cudaTypedefs.h>
+
+#include <climits>
 
 #include "fdc_attn_common.cuh"
 
@@ -27,15 +33,19 @@ using namespace fdc;
 
 namespace {
 
-constexpr int TILE = FDC_TILE_ROWS;          // KV rows per tile = N of the QK MMA, K of the PV MMA
-constexpr int MROWS = 128;                   // M of both MMAs (query rows, zero padded)
+constexpr int D = 128;                       // head_dim handled by this kernel
+constexpr int TILE = FDC_TILE_ROWS;          // rows per entry of the visited-tile list
+constexpr int RROWS = 2 * TILE;              // KV rows per round = M of S^T = K of O^T
 constexpr int NSOFT = 8;                     // softmax warps
-constexpr int W_KPROD = 8, W_MMA = 9, W_VPROD = 10;
-constexpr int THREADS = 352;
-constexpr int NSBUF = 4;                     // score buffers in TMEM: S = Q K^T runs up to 4 tiles ahead
-constexpr uint32_t TMEM_COLS = 512;          // S0..S3 [0,256) | O [256, 256 + head_dim)
-constexpr int MAXRING = 8;                   // stages per ring (K ring, V ring)
-constexpr float RESCALE_LOG2 = 8.f;
+constexpr int W_KPROD = 8, W_MMA = 9, W_VPROD = 10, W_VFIX = 11;
+constexpr int THREADS = 384;
+constexpr uint32_t TMEM_COLS = 512;          // S^T 0 [0,128) | S^T 1 [128,256) | O^T [256,384)
+constexpr uint32_t TM_O = 256;
+constexpr int PANEL = RROWS * 128;           // 128 rows x 128 bytes (64 bf16 columns)
+constexpr int STAGE = (D / 64) * PANEL;      // one K (or V) stage: 128 rows x head_dim
+constexpr int MAXST = 4;                     // stages per ring at most
+constexpr float RAISE_LOG2 = 8.f;
+constexpr float UNSET = 1.0e30f;             // -reference of a column that has seen nothing yet
 
 // ---------------------------------------------------------------- tcgen05 wrappers
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -44,15 +54,18 @@ __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.a
 
 // Shared-memory matrix descriptor (128-byte swizzle, descriptor version 1): start address,
 // leading-dimension byte offset, stride-dimension byte offset, all in units of 16 bytes.
+// K-major operand: SBO = distance of 8-row groups.  MN-major operand: LBO = distance of
+// 64-element groups along M/N, SBO = distance of 8-row groups along K.
 __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes)
 {
     return (uint64_t)((addr >> 4) & 0x3FFFu) | ((uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16) |
            ((uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32) | (1ull << 46) | (2ull << 61);
 }
-// Instruction descriptor of kind::f16: fp32 accumulate, bf16 A and B, M x N, B optionally MN-major.
-__device__ __forceinline__ uint32_t instr_desc(int m, int n, int b_mn_major)
+// Instruction descriptor of kind::f16: fp32 accumulate, bf16 A and B, M x N; mn_major = 1 makes
+// BOTH operands MN-major (contiguous along M resp. N), 0 makes both K-major.
+__device__ __forceinline__ uint32_t instr_desc(int m, int n, uint32_t mn_major)
 {
-    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)b_mn_major << 16) | ((uint32_t)(n >> 3) << 17) |
+    return (1u << 4) | (1u << 7) | (1u << 10) | (mn_major << 15) | (mn_major << 16) | ((uint32_t)(n >> 3) << 17) |
            ((uint32_t)(m >> 4) << 24);
 }
 __device__ __forceinline__ void umma(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate)
@@ -70,42 +83,48 @@ __device__ __forceinline__ void umma_commit(uint32_t bar)
 
 #define FDC_R8(v, o) "=r"(v[o + 0]), "=r"(v[o + 1]), "=r"(v[o + 2]), "=r"(v[o + 3]), "=r"(v[o + 4]), "=r"(v[o + 5]), "=r"(v[o + 6]), "=r"(v[o + 7])
 #define FDC_I8(v, o) "r"(v[o + 0]), "r"(v[o + 1]), "r"(v[o + 2]), "r"(v[o + 3]), "r"(v[o + 4]), "r"(v[o + 5]), "r"(v[o + 6]), "r"(v[o + 7])
-// 32 consecutive fp32 columns of this thread's TMEM lane.
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32])
+// N consecutive fp32 columns of this thread's TMEM lane (N = 8, 16 or 32).
+template <int N>
+__device__ __forceinline__ void tmem_ld(uint32_t taddr, uint32_t (&v)[N])
 {
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,"
-        "%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
-        : FDC_R8(v, 0), FDC_R8(v, 8), FDC_R8(v, 16), FDC_R8(v, 24)
-        : "r"(taddr)
-        : "memory");
+    static_assert(N == 8 || N == 16 || N == 32, "column count");
+    if constexpr (N == 32) {
+        asm volatile(
+            "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,"
+            "%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+            : FDC_R8(v, 0), FDC_R8(v, 8), FDC_R8(v, 16), FDC_R8(v, 24)
+            : "r"(taddr)
+            : "memory");
+    } else if constexpr (N == 16) {
+        asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+                     : FDC_R8(v, 0), FDC_R8(v, 8)
+                     : "r"(taddr)
+                     : "memory");
+    } else {
+        asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];" : FDC_R8(v, 0) : "r"(taddr) : "memory");
+    }
 }
-__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&v)[32])
+template <int N>
+__device__ __forceinline__ void tmem_st(uint32_t taddr, const uint32_t (&v)[N])
 {
-    asm volatile(
-        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%32], {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,"
-        "%24,%25,%26,%27,%28,%29,%30,%31};"
-        ::FDC_I8(v, 0), FDC_I8(v, 8), FDC_I8(v, 16), FDC_I8(v, 24), "r"(taddr)
-        : "memory");
+    static_assert(N == 8 || N == 16 || N == 32, "column count");
+    if constexpr (N == 32) {
+        asm volatile(
+            "tcgen05.st.sync.aligned.32x32b.x32.b32 [%32], {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,"
+            "%24,%25,%26,%27,%28,%29,%30,%31};"
+            ::FDC_I8(v, 0), FDC_I8(v, 8), FDC_I8(v, 16), FDC_I8(v, 24), "r"(taddr)
+            : "memory");
+    } else if constexpr (N == 16) {
+        asm volatile("tcgen05.st.sync.aligned.32x32b.x16.b32 [%16], {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15};"
+                     ::FDC_I8(v, 0), FDC_I8(v, 8), "r"(taddr)
+                     : "memory");
+    } else {
+        asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%8], {%0,%1,%2,%3,%4,%5,%6,%7};" ::FDC_I8(v, 0), "r"(taddr) : "memory");
+    }
 }
-__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&v)[32])
-{
-    asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
-                 : FDC_R8(v, 0), FDC_R8(v, 8)
-                 : "r"(taddr)
-                 : "memory");
-}
-__device__ __forceinline__ void tmem_ld8(uint32_t taddr, uint32_t (&v)[32])
-{
-    asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];" : FDC_R8(v, 0) : "r"(taddr) : "memory");
-}
-template <int WS>
-__device__ __forceinline__ void tmem_ld_slice(uint32_t taddr, uint32_t (&v)[32])
-{
-    if constexpr (WS == 32) tmem_ld32(taddr, v);
-    else if constexpr (WS == 16) tmem_ld16(taddr, v);
-    else tmem_ld8(taddr, v);
-}
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
 // OR of a predicate over the softmax threads (named barrier 1)
 __device__ __forceinline__ bool soft_any(bool x)
 {
@@ -117,43 +136,44 @@ __device__ __forceinline__ bool soft_any(bool x)
     return out != 0;
 }
 __device__ __forceinline__ void soft_sync() { asm volatile("bar.sync 1, %0;" ::"n"(NSOFT * 32) : "memory"); }
-__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
 __device__ __forceinline__ uint32_t pack2(float lo, float hi)
 {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t*>(&v);
 }
-
-template <int D>
-struct Smem {
-    static constexpr int KV_PANEL = TILE * 128;               // 64 rows x 128 bytes
-    static constexpr int KV_BYTES = TILE * D * 2;             // one K (or V) tile = one ring stage
-    static constexpr int Q_PANEL = MROWS * 128;
-    static constexpr int Q_BYTES = MROWS * D * 2;
-    static constexpr int P_BYTES = MROWS * TILE * 2;          // one P buffer: 128 rows x 128 bytes
-};
+// Monotone map float -> int (for integer max reductions).
+__device__ __forceinline__ int ord_of(float x)
+{
+    const int i = __float_as_int(x);
+    return i ^ ((i >> 31) & 0x7fffffff);
+}
+__device__ __forceinline__ float ord_to(int i) { return __int_as_float(i ^ ((i >> 31) & 0x7fffffff)); }
 
 // Everything a role needs to find its barriers and buffers.
 struct Ctx {
-    uint32_t k_full, k_empty, v_full, v_empty, s_full, p_full, pv_done, q_ready, o_free;
-    uint32_t tm_s, tm_o;
+    uint32_t k_full, k_empty, v_full, v_empty, v_clean, s_full, p_full, pv_done, q_ready, o_free;
+    uint32_t tmem;
     unsigned char *kring, *vring, *qs, *ps;
-    float* xch;
+    float *mneg, *alpha, *lred;      // [128] -reference per column, [128] rescale factors, [4][128] partial sums
+    int *cmax, *flags;               // [128] column maxima (ordered ints), [2] flags of the raise path
     int* pre;
     volatile int* abortp;
-    int nk, nv;
+    int nk, nv, q_panel, p_buf, npb; // ring depths, bytes per 64-column panel of Q^T, bytes per P^T buffer, P^T buffers (1 or 2)
 };
 
-// One TMA producer warp: streams the K (or V) tiles of this CTA's units into its ring.
-template <int D>
+// A round: up to two entries of a segment's tile list.
+struct Round {
+    int nt, tile0, tile1;
+};
+
+// One TMA producer warp: streams the K (or V) tiles of this CTA's units into its ring, two tiles
+// per stage (rows 0-63 and 64-127 of both 64-column panels).
 __device__ __forceinline__ void producer_loop(const AttnParams& p, const Ctx& cx, const CUtensorMap* tm, unsigned char* ring,
                                               uint32_t full, uint32_t empty, int nst, long long lo, long long hi, int lane)
 {
-    using L = Smem<D>;
     int s = 0;
-    uint32_t it = 0;
+    uint32_t g = 0;
     long long u = lo;
     int ok = 1;
     while (u < hi && ok) {
@@ -161,18 +181,22 @@ __device__ __forceinline__ void producer_loop(const AttnParams& p, const Ctx& cx
         for (int jb = sg.j0; jb < sg.j1 && ok; jb += 32) {
             const int jn = sg.j1 - jb < 32 ? sg.j1 - jb : 32;
             const int my_tile = lane < jn ? p.tiles[(size_t)sg.s * p.ntile_max + jb + lane] : 0;
-            for (int k = 0; k < jn && ok; ++k, ++it) {
-                const int tile = __shfl_sync(0xffffffffu, my_tile, k);
+            for (int k = 0; k < jn && ok; k += 2, ++g) {
+                const int nt = jn - k < 2 ? 1 : 2;
+                const int t0 = __shfl_sync(0xffffffffu, my_tile, k);
+                const int t1 = __shfl_sync(0xffffffffu, my_tile, (k + 1) & 31);
                 if (lane == 0) {
-                    const int st = it % nst;
-                    if (!mbar_wait(empty + 8 * st, ((it / nst) & 1) ^ 1, cx.abortp, p.status)) {
+                    const int st = g % nst;
+                    if (!mbar_wait(empty + 8 * st, ((g / nst) & 1) ^ 1, cx.abortp, p.status)) {
                         ok = 0;
                     } else {
-                        const uint32_t dst = smem_u32(ring + (size_t)st * L::KV_BYTES);
-                        mbar_expect_tx(full + 8 * st, L::KV_BYTES);
+                        const uint32_t dst = smem_u32(ring + (size_t)st * STAGE);
+                        mbar_expect_tx(full + 8 * st, nt * (STAGE / 2));
 #pragma unroll
-                        for (int h = 0; h < D / 64; ++h)
-                            tma_load_4d(dst + h * L::KV_PANEL, tm, full + 8 * st, h * 64, tile * TILE, sg.g, sg.s);
+                        for (int h = 0; h < D / 64; ++h) {
+                            tma_load_4d(dst + h * PANEL, tm, full + 8 * st, h * 64, t0 * TILE, sg.g, sg.s);
+                            if (nt == 2) tma_load_4d(dst + h * PANEL + TILE * 128, tm, full + 8 * st, h * 64, t1 * TILE, sg.g, sg.s);
+                        }
                     }
                 }
                 ok = __shfl_sync(0xffffffffu, ok, 0);
@@ -182,201 +206,307 @@ __device__ __forceinline__ void producer_loop(const AttnParams& p, const Ctx& cx
     }
     if (!ok && lane == 0) {
         // give the copies already in flight a bounded chance to land before the CTA ends
-        const uint32_t first = it > (uint32_t)nst ? it - nst : 0;
-        for (uint32_t k = first; k < it; ++k) {
+        const uint32_t first = g > (uint32_t)nst ? g - nst : 0;
+        for (uint32_t k = first; k < g; ++k) {
             const uint32_t bar = full + 8 * (k % nst), ph = (k / nst) & 1;
             for (uint32_t i = 0; i < (1u << 16) && !mbar_try(bar, ph); ++i) __nanosleep(64);
         }
     }
 }
 
-// The MMA issuer thread.
-template <int D>
-__device__ __forceinline__ void mma_loop(const AttnParams& p, const Ctx& cx, long long lo, long long hi)
+// Warp 11: V rows that are invisible to every branch of the scene are cleared in shared memory
+// before the stage is released to O^T += V^T P^T (their P column is exactly 0, but the row may
+// hold NaN or Inf).  Stages wholly inside the prefix are released as they are.
+__device__ __forceinline__ void vfix_loop(const AttnParams& p, const Ctx& cx, long long lo, long long hi, int lane)
 {
-    using L = Smem<D>;
-    const uint32_t idesc_qk = instr_desc(MROWS, TILE, 0), idesc_pv = instr_desc(MROWS, D, 1);
-    const uint64_t q_desc = smem_desc(smem_u32(cx.qs), 16, 1024);
-    const uint64_t p_desc = smem_desc(smem_u32(cx.ps), 16, 1024);
-    const uint64_t k_desc0 = smem_desc(smem_u32(cx.kring), 16, 1024);
-    const uint64_t v_desc0 = smem_desc(smem_u32(cx.vring), L::KV_PANEL, 1024);
-    auto issue_qk = [&](uint32_t g) -> bool {
-        const int st = g % cx.nk;
-        if (!mbar_wait(cx.k_full + 8 * st, (g / cx.nk) & 1, cx.abortp, p.status)) return false;
-        tc_fence_after();
-        const uint64_t kd = k_desc0 + (uint64_t)((st * L::KV_BYTES) >> 4);
-#pragma unroll
-        for (int ks = 0; ks < D / 16; ++ks)
-            umma(cx.tm_s + (g & (NSBUF - 1)) * TILE, q_desc + (uint64_t)(((ks >> 2) * L::Q_PANEL + (ks & 3) * 32) >> 4),
-                 kd + (uint64_t)(((ks >> 2) * L::KV_PANEL + (ks & 3) * 32) >> 4), idesc_qk, ks > 0);
-        umma_commit(cx.k_empty + 8 * st);
-        umma_commit(cx.s_full + 8 * (g & (NSBUF - 1)));
-        return true;
-    };
     int s = 0;
-    uint32_t it = 0, seg = 0;
+    uint32_t g = 0;
     long long u = lo;
-    bool ok = true;
+    int ok = 1;
     while (u < hi && ok) {
         const Segment sg = decode_segment(u, hi, cx.pre, p.hkv, s);
-        const int n = sg.j1 - sg.j0;
-        ok = mbar_wait(cx.q_ready, seg & 1, cx.abortp, p.status);
-        for (int a = 0; a < NSBUF && a < n && ok; ++a) ok = issue_qk(it + a);
-        for (int t = 0; t < n && ok; ++t) {
-            const uint32_t g = it + t;
-            ok = mbar_wait(cx.p_full + 8 * (g & 1), (g >> 1) & 1, cx.abortp, p.status);
-            if (ok && t == 0 && seg > 0) ok = mbar_wait(cx.o_free, (seg - 1) & 1, cx.abortp, p.status);
-            const int st = g % cx.nv;
-            if (ok) ok = mbar_wait(cx.v_full + 8 * st, (g / cx.nv) & 1, cx.abortp, p.status);
-            if (!ok) break;
-            tc_fence_after();
-            const uint64_t vd = v_desc0 + (uint64_t)((st * L::KV_BYTES) >> 4);
-            const uint64_t pd = p_desc + (uint64_t)(((g & 1) * L::P_BYTES) >> 4);
-#pragma unroll
-            for (int kk = 0; kk < TILE / 16; ++kk)
-                umma(cx.tm_o, pd + (uint64_t)((kk * 32) >> 4), vd + (uint64_t)((kk * 2048) >> 4), idesc_pv, (t > 0 || kk > 0) ? 1u : 0u);
-            umma_commit(cx.v_empty + 8 * st);
-            umma_commit(cx.pv_done + 8 * (g & 1));
-            if (t + NSBUF < n) ok = issue_qk(g + NSBUF);
+        const int A = p.n_active[sg.s];
+        for (int jb = sg.j0; jb < sg.j1 && ok; jb += 32) {
+            const int jn = sg.j1 - jb < 32 ? sg.j1 - jb : 32;
+            const int my_tile = lane < jn ? p.tiles[(size_t)sg.s * p.ntile_max + jb + lane] : 0;
+            for (int k = 0; k < jn && ok; k += 2, ++g) {
+                const int nt = jn - k < 2 ? 1 : 2;
+                const int st = g % cx.nv;
+                int okw = 1;
+                if (lane == 0) okw = mbar_wait(cx.v_full + 8 * st, (g / cx.nv) & 1, cx.abortp, p.status);
+                ok = __shfl_sync(0xffffffffu, okw, 0);
+                if (!ok) break;
+                unsigned char* vs = cx.vring + (size_t)st * STAGE;
+                bool touched = false;
+                for (int i = 0; i < nt; ++i) {
+                    const int tile = __shfl_sync(0xffffffffu, my_tile, (k + i) & 31);
+                    if (tile * TILE + TILE <= p.P) continue;                 // all rows visible to everybody
+                    uint64_t um = 0ull;
+                    for (int b = lane; b < A; b += 32)
+                        um |= tile_rowmask(p.mask + ((size_t)sg.s * p.max_active + b) * p.W, p.W, p.P, tile);
+                    const uint32_t ul = __reduce_or_sync(0xffffffffu, (uint32_t)um);
+                    const uint32_t uh = __reduce_or_sync(0xffffffffu, (uint32_t)(um >> 32));
+                    uint64_t z = ~(((uint64_t)uh << 32) | ul);
+                    // two rows per step: lanes 0-15 clear one row (2 panels x 8 chunks of 16 bytes), lanes 16-31 the next
+                    while (z) {
+                        const int r0 = __ffsll((long long)z) - 1;
+                        z &= z - 1;
+                        int r1 = -1;
+                        if (z) {
+                            r1 = __ffsll((long long)z) - 1;
+                            z &= z - 1;
+                        }
+                        const int r = lane < 16 ? r0 : r1;
+                        if (r >= 0) {
+                            const int l16 = lane & 15;
+                            *reinterpret_cast<uint4*>(vs + (l16 >> 3) * PANEL + (i * TILE + r) * 128 + ((l16 & 7) << 4)) =
+                                make_uint4(0u, 0u, 0u, 0u);
+                        }
+                        touched = true;
+                    }
+                }
+                if (touched) fence_async_smem();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(cx.v_clean + 8 * st);
+            }
         }
-        it += n;
+        u = sg.next_u;
+    }
+}
+
+// The MMA issuer (whole warp follows the loop, lane 0 waits and issues).
+__device__ __forceinline__ void mma_loop(const AttnParams& p, const Ctx& cx, long long lo, long long hi, int lane)
+{
+    const uint64_t q_desc = smem_desc(smem_u32(cx.qs), 16, 1024);
+    const uint64_t k_desc0 = smem_desc(smem_u32(cx.kring), 16, 1024);
+    const uint64_t v_desc0 = smem_desc(smem_u32(cx.vring), PANEL, 1024);
+    const uint64_t p_desc0 = smem_desc(smem_u32(cx.ps), PANEL, 1024);
+    const uint32_t tm_o = cx.tmem + TM_O;
+    int s = 0;
+    uint32_t g0 = 0, seg = 0;
+    long long u = lo;
+    int ok = 1;
+    while (u < hi && ok) {
+        const Segment sg = decode_segment(u, hi, cx.pre, p.hkv, s);
+        const int ntile = sg.j1 - sg.j0;
+        const int nr = (ntile + 1) >> 1;
+        if (lane == 0) {
+            int M = p.n_active[sg.s] * p.group;
+            const int NP = M <= 16 ? 16 : (M <= 32 ? 32 : (M <= 64 ? 64 : 128));
+            const uint32_t idesc_qk = instr_desc(RROWS, NP, 0), idesc_pv = instr_desc(D, NP, 1);
+            // S^T[g & 1] = K(stage) Q^T
+            auto issue_qk = [&](uint32_t g) -> bool {
+                const int st = g % cx.nk;
+                if (!mbar_wait(cx.k_full + 8 * st, (g / cx.nk) & 1, cx.abortp, p.status)) return false;
+                tc_fence_after();
+                const uint64_t kd = k_desc0 + (uint64_t)((st * STAGE) >> 4);
+#pragma unroll
+                for (int ks = 0; ks < D / 16; ++ks)
+                    umma(cx.tmem + (g & 1) * 128, kd + (uint64_t)(((ks >> 2) * PANEL + (ks & 3) * 32) >> 4),
+                         q_desc + (uint64_t)(((ks >> 2) * cx.q_panel + (ks & 3) * 32) >> 4), idesc_qk, ks > 0);
+                umma_commit(cx.k_empty + 8 * st);
+                umma_commit(cx.s_full + 8 * (g & 1));
+                return true;
+            };
+            bool good = mbar_wait(cx.q_ready, seg & 1, cx.abortp, p.status);
+            for (int a = 0; a < 2 && a < nr && good; ++a) good = issue_qk(g0 + a);
+            for (int t = 0; t < nr && good; ++t) {
+                const uint32_t g = g0 + t;
+                const int rows = (t == nr - 1 && (ntile & 1)) ? TILE : RROWS;
+                good = mbar_wait(cx.p_full + 8 * (g & 1), (g >> 1) & 1, cx.abortp, p.status);
+                if (good && t == 0 && seg > 0) good = mbar_wait(cx.o_free, (seg - 1) & 1, cx.abortp, p.status);
+                const int st = g % cx.nv;
+                if (good) good = mbar_wait(cx.v_clean + 8 * st, (g / cx.nv) & 1, cx.abortp, p.status);
+                if (!good) break;
+                tc_fence_after();
+                const uint64_t vd = v_desc0 + (uint64_t)((st * STAGE) >> 4);
+                const uint64_t pd = p_desc0 + (uint64_t)((((g & 1) & (cx.npb - 1)) * cx.p_buf) >> 4);
+                for (int kk = 0; kk < rows / 16; ++kk)
+                    umma(tm_o, vd + (uint64_t)((kk * 2048) >> 4), pd + (uint64_t)((kk * 2048) >> 4), idesc_pv, (t > 0 || kk > 0) ? 1u : 0u);
+                umma_commit(cx.v_empty + 8 * st);
+                umma_commit(cx.pv_done + 8 * (g & 1));
+                if (t + 2 < nr) good = issue_qk(g + 2);
+            }
+            ok = good;
+        }
+        ok = __shfl_sync(0xffffffffu, ok, 0);
+        g0 += nr;
         ++seg;
         u = sg.next_u;
     }
 }
 
-// The softmax warps' work on one segment; WS = score columns per thread (64 / threads per row).
-template <int D, int WS>
-__device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& cx, const Segment& sg, uint32_t& it, bool& dead,
+// The softmax warps' work on one segment; NPH = query columns per thread (half of NP).
+template <int NPH>
+__device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& cx, const Segment& sg, uint32_t& g, bool& dead,
                                                 const int warp, const int lane)
 {
-    using L = Smem<D>;
-    constexpr int NSLICE = TILE / WS;             // threads sharing one query row
-    constexpr int MP = MROWS * 2 / NSLICE;        // rows per replica
+    constexpr int NP = 2 * NPH;
+    constexpr int CH = NPH < 32 ? NPH : 32;       // columns handled at a time
+    constexpr int NCH = NPH / CH;
+    const int tid = threadIdx.x;                  // 0..255
     const int q4 = warp & 3, half = warp >> 2;
-    const int i_row = q4 * 32 + lane;             // MMA row = TMEM lane of this thread
+    const int krow = q4 * 32 + lane;              // KV row of the round = TMEM lane of S^T; head_dim index for O^T
     const uint32_t lane_base = (uint32_t)(q4 * 32) << 16;
+    const int col0 = half * NPH;
     const float c = p.scale_log2;
     const int A = p.n_active[sg.s];
     const int M = A * p.group;
-    const int m = i_row & (MP - 1);               // query row of this thread
-    const int sigma = (i_row / MP) * 2 + half;    // its column slice
-    const int col0 = sigma * WS;
-    const bool row_on = m < M;
-    const bool warp_on = ((q4 * 32) & (MP - 1)) < M;      // some lane of the warp has a live row
-    const bool owner = half == 0 && q4 * 32 < MP;         // warp whose TMEM lanes are the rows of replica 0
-    const int br = row_on ? m / p.group : 0;
-    const uint64_t* mrow = p.mask + ((size_t)sg.s * p.max_active + br) * p.W;
+    const int G = p.group;
     auto wait_u = [&](uint32_t bar, uint32_t parity) {    // warp-uniform outcome
         if (!dead && !mbar_wait(bar, parity, cx.abortp, p.status)) dead = true;
         dead = __any_sync(0xffffffffu, dead);
     };
-    // the query tile (A operand of S = Q K^T): MMA row i holds query row i mod MP; K-major, 128B swizzle
-    if (!dead) {
-        const uint4* src = reinterpret_cast<const uint4*>(
-            reinterpret_cast<const __nv_bfloat16*>(p.q) +
-            (((size_t)sg.s * p.max_active + br) * p.hq + (size_t)sg.g * p.group + (m - br * p.group)) * D);
-#pragma unroll
-        for (int cc = 0; cc < D / 16; ++cc) {
-            const int ch = half * (D / 16) + cc;
-            const uint4 v = row_on ? src[ch] : make_uint4(0u, 0u, 0u, 0u);
-            *reinterpret_cast<uint4*>(cx.qs + (ch >> 3) * L::Q_PANEL + i_row * 128 + (((ch & 7) ^ (i_row & 7)) << 4)) = v;
+    // ---- Q^T (B operand of S^T = K Q^T): row n = query row, K-major, 128B swizzle, rows >= M zero
+    {
+        const uint4* qg = reinterpret_cast<const uint4*>(p.q);
+        for (int idx = tid; idx < NP * (D / 8); idx += NSOFT * 32) {
+            const int n = idx / (D / 8), ch = idx - n * (D / 8);
+            uint4 v = make_uint4(0u, 0u, 0u, 0u);
+            if (n < M) {
+                const int b = n / G, hg = n - b * G;
+                v = qg[((((size_t)sg.s * p.max_active + b) * p.hq + (size_t)sg.g * G + hg) * D) / 8 + ch];
+            }
+            *reinterpret_cast<uint4*>(cx.qs + (ch >> 3) * cx.q_panel + n * 128 + (((ch & 7) ^ (n & 7)) << 4)) = v;
+        }
+        if (tid < NP) {
+            cx.mneg[tid] = UNSET;
+            cx.cmax[tid] = INT_MIN;
         }
         fence_async_smem();
-        mbar_arrive(cx.q_ready);
+        if (!dead) mbar_arrive(cx.q_ready);
+        soft_sync();
     }
-    float ms = -INFINITY, l = 0.f;        // row reference maximum (scaled log2 units), this thread's partial sum
-    const int n = sg.j1 - sg.j0;
-    for (int jb = 0; jb < n; jb += 32) {
-        const int jn = n - jb < 32 ? n - jb : 32;
+    float l[NPH];
+#pragma unroll
+    for (int i = 0; i < NPH; ++i) l[i] = 0.f;
+
+    const int ntile = sg.j1 - sg.j0;
+    int t = 0;                                    // round within the segment
+    for (int jb = 0; jb < ntile; jb += 32) {
+        const int jn = ntile - jb < 32 ? ntile - jb : 32;
         const int my_tile = lane < jn ? p.tiles[(size_t)sg.s * p.ntile_max + sg.j0 + jb + lane] : 0;
-        for (int k = 0; k < jn; ++k, ++it) {
-            const int tile = __shfl_sync(0xffffffffu, my_tile, k);
-            const int t = jb + k;
-            const uint32_t b = it & 1, sb = it & (NSBUF - 1);
-            const bool masked = tile * TILE + TILE > p.P;
-            wait_u(cx.s_full + 8 * sb, (it / NSBUF) & 1);
+        for (int k = 0; k < jn; k += 2, ++g, ++t) {
+            const int nt = jn - k < 2 ? 1 : 2;
+            const uint32_t b = g & 1;
+            const int ti = q4 >> 1;                                   // which tile of the round this warp's rows are in
+            const int tile = __shfl_sync(0xffffffffu, my_tile, (k + ti) & 31);
+            const bool live = ti < nt && !dead;                       // rows 64..127 of a one-tile round hold nothing
+            const bool masked = live && tile * TILE + TILE > p.P;
+            // visibility of this warp's 32 rows for branch `lane` (and `lane + 32`), Eq. 1
+            uint32_t wlo = 0xffffffffu, whi = 0xffffffffu;
+            if (masked) {
+                uint64_t m0 = 0ull, m1 = 0ull;
+                if (lane < A) m0 = tile_rowmask(p.mask + ((size_t)sg.s * p.max_active + lane) * p.W, p.W, p.P, tile);
+                if (lane + 32 < A) m1 = tile_rowmask(p.mask + ((size_t)sg.s * p.max_active + lane + 32) * p.W, p.W, p.P, tile);
+                wlo = (q4 & 1) ? (uint32_t)(m0 >> 32) : (uint32_t)m0;
+                whi = (q4 & 1) ? (uint32_t)(m1 >> 32) : (uint32_t)m1;
+            }
+            wait_u(cx.s_full + 8 * b, (g >> 1) & 1);
             tc_fence_after();
-            if (masked && !dead) {
-                // rows no branch may see can hold anything: clear their V so that 0 * NaN cannot arise
-                wait_u(cx.v_full + 8 * (it % cx.nv), (it / cx.nv) & 1);
-                uint64_t um = 0ull;
-                for (int bb = lane; bb < A; bb += 32)
-                    um |= tile_rowmask(p.mask + ((size_t)sg.s * p.max_active + bb) * p.W, p.W, p.P, tile);
-                const uint32_t ul = __reduce_or_sync(0xffffffffu, (uint32_t)um);
-                const uint32_t uh = __reduce_or_sync(0xffffffffu, (uint32_t)(um >> 32));
-                uint64_t z = ~(((uint64_t)uh << 32) | ul);
-                unsigned char* vs = cx.vring + (size_t)(it % cx.nv) * L::KV_BYTES;
-                while (z && !dead) {
-                    const int zr = __ffsll((long long)z) - 1;
-                    z &= z - 1;
-                    if ((zr & 7) != warp) continue;
-                    for (int i = lane; i < D / 4; i += 32) {
-                        const int ch = i >> 1;
-                        *reinterpret_cast<uint2*>(vs + (ch >> 3) * L::KV_PANEL + zr * 128 + (((ch & 7) ^ (zr & 7)) << 4) + (i & 1) * 8) =
-                            make_uint2(0u, 0u);
-                    }
-                }
-            }
-            uint32_t sv[32];
-            float mx = -INFINITY;
-            const bool work = warp_on && !dead;
-            if (work) {
-                tmem_ld_slice<WS>(cx.tm_s + lane_base + sb * TILE + col0, sv);
+            const uint32_t s_addr = cx.tmem + lane_base + b * 128 + col0;
+            // args[i] = score * scale * log2(e) - reference, -inf where Eq. 1 hides the row
+            auto load_args = [&](int chunk, uint32_t (&sv)[CH], bool minus_ref) {
+                tmem_ld<CH>(s_addr + chunk * CH, sv);
                 tmem_wait_ld();
-                uint32_t vis = row_on ? 0xffffffffu : 0u;
-                if (masked && row_on) vis = (uint32_t)(tile_rowmask(mrow, p.W, p.P, tile) >> col0);
+                int bq = (col0 + chunk * CH) / G, rem = (col0 + chunk * CH) - bq * G;
 #pragma unroll
-                for (int i = 0; i < WS; ++i) {
-                    const float x = ((vis >> i) & 1) ? __uint_as_float(sv[i]) * c : -INFINITY;
-                    sv[i] = __float_as_uint(x);
-                    mx = fmaxf(mx, x);
+                for (int i = 0; i < CH; ++i) {
+                    float a = minus_ref ? fmaf(__uint_as_float(sv[i]), c, cx.mneg[col0 + chunk * CH + i]) : __uint_as_float(sv[i]) * c;
+                    if (masked) {
+                        const uint32_t bits = __shfl_sync(0xffffffffu, bq < 32 ? wlo : whi, bq & 31);
+                        if (!((bits >> lane) & 1)) a = -INFINITY;
+                        if (++rem == G) {
+                            rem = 0;
+                            ++bq;
+                        }
+                    }
+                    sv[i] = __float_as_uint(a);
+                }
+            };
+            uint32_t sv[CH];
+            float amax = -INFINITY;
+            if (live) {
+#pragma unroll
+                for (int ch = 0; ch < NCH; ++ch) {
+                    load_args(ch, sv, true);
+#pragma unroll
+                    for (int i = 0; i < CH; ++i) amax = fmaxf(amax, __uint_as_float(sv[i]));
                 }
             }
-            // does any row need a higher reference?  (first visible score, or a jump of more than 2^8)
-            const bool flag = work && (ms == -INFINITY ? mx != -INFINITY : mx > ms + RESCALE_LOG2);
-            if (soft_any(flag)) {
-                cx.xch[m * NSLICE + sigma] = mx;
-                soft_sync();
-                float mr = -INFINITY;
+            // does some column need a (higher) reference?  first visible score, or a jump of more than 2^8
+            if (soft_any(live && amax > RAISE_LOG2)) {
+                if (live) {
 #pragma unroll
-                for (int j = 0; j < NSLICE; ++j) mr = fmaxf(mr, cx.xch[m * NSLICE + j]);
-                const bool first = ms == -INFINITY && mr != -INFINITY;
-                const bool jump = ms != -INFINITY && mr > ms + RESCALE_LOG2;
-                const float alpha = jump ? fast_exp2(ms - mr) : 1.f;
-                l *= alpha;
-                if (owner && t > 0 && __any_sync(0xffffffffu, jump && work)) {
-                    // O must not be written by an MMA while it is rescaled: the previous PV has to be complete
-                    wait_u(cx.pv_done + 8 * ((it - 1) & 1), ((it - 1) >> 1) & 1);
-                    tc_fence_after();
-                    if (!dead) {
+                    for (int ch = 0; ch < NCH; ++ch) {
+                        load_args(ch, sv, false);
 #pragma unroll
-                        for (int cc = 0; cc < D / 32; ++cc) {
-                            uint32_t ov[32];
-                            tmem_ld32(cx.tm_o + lane_base + cc * 32, ov);
-                            tmem_wait_ld();
-#pragma unroll
-                            for (int i = 0; i < 32; ++i) ov[i] = __float_as_uint(__uint_as_float(ov[i]) * alpha);
-                            tmem_st32(cx.tm_o + lane_base + cc * 32, ov);
+                        for (int i = 0; i < CH; ++i) {
+                            const int wm = __reduce_max_sync(0xffffffffu, ord_of(__uint_as_float(sv[i])));
+                            if (lane == 0) atomicMax(&cx.cmax[col0 + ch * CH + i], wm);
                         }
-                        tmem_wait_st();
                     }
                 }
-                if (first || jump) ms = mr;
+                if (tid == 0) cx.flags[0] = 0;
+                soft_sync();
+                if (tid < NP) {
+                    const float mr = ord_to(cx.cmax[tid]);
+                    const float old = cx.mneg[tid];                    // -reference, or UNSET
+                    float al = 1.f;
+                    if (old == UNSET) {
+                        if (mr != -INFINITY) cx.mneg[tid] = -mr;
+                    } else if (mr > RAISE_LOG2 - old) {
+                        al = fast_exp2(-old - mr);
+                        cx.mneg[tid] = -mr;
+                        cx.flags[0] = 1;
+                    }
+                    cx.alpha[tid] = al;
+                    cx.cmax[tid] = INT_MIN;
+                }
+                soft_sync();
+                if (cx.flags[0]) {                                     // a reference moved: rescale sums and accumulator
+#pragma unroll
+                    for (int i = 0; i < NPH; ++i) l[i] *= cx.alpha[col0 + i];
+                    if (t > 0) {
+                        wait_u(cx.pv_done + 8 * ((g - 1) & 1), ((g - 1) >> 1) & 1);   // no MMA may be writing O^T
+                        tc_fence_after();
+                        if (!dead) {
+#pragma unroll
+                            for (int ch = 0; ch < NCH; ++ch) {
+                                uint32_t ov[CH];
+                                tmem_ld<CH>(cx.tmem + lane_base + TM_O + col0 + ch * CH, ov);
+                                tmem_wait_ld();
+#pragma unroll
+                                for (int i = 0; i < CH; ++i) ov[i] = __float_as_uint(__uint_as_float(ov[i]) * cx.alpha[col0 + ch * CH + i]);
+                                tmem_st<CH>(cx.tmem + lane_base + TM_O + col0 + ch * CH, ov);
+                            }
+                            tmem_wait_st();
+                        }
+                    }
+                }
+                if (NCH == 1 && live) load_args(0, sv, true);
             }
-            // P[b] is still being read until the PV of two tiles ago has completed
-            wait_u(cx.pv_done + 8 * b, ((it >> 1) & 1) ^ 1);
-            if (work && !dead) {
-                const float mref = ms == -INFINITY ? 0.f : ms;
-                unsigned char* prow = cx.ps + b * L::P_BYTES + m * 128;
+            // the P^T buffer is still being read until the PV that used it last (two rounds ago, or
+            // the previous round when there is a single buffer) has completed
+            if (cx.npb == 2) wait_u(cx.pv_done + 8 * b, ((g >> 1) & 1) ^ 1);
+            else if (g > 0) wait_u(cx.pv_done + 8 * ((g - 1) & 1), ((g - 1) >> 1) & 1);
+            if (live) {
+                unsigned char* prow = cx.ps + (b & (cx.npb - 1)) * cx.p_buf + krow * 128;
 #pragma unroll
-                for (int ch = 0; ch < WS / 8; ++ch) {
-                    float e[8];
+                for (int ch = 0; ch < NCH; ++ch) {
+                    if (NCH > 1) load_args(ch, sv, true);
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) e[i] = fast_exp2(__uint_as_float(sv[ch * 8 + i]) - mref);
-                    l += ((e[0] + e[1]) + (e[2] + e[3])) + ((e[4] + e[5]) + (e[6] + e[7]));
-                    *reinterpret_cast<uint4*>(prow + ((((col0 >> 3) + ch) ^ (m & 7)) << 4)) =
-                        make_uint4(pack2(e[0], e[1]), pack2(e[2], e[3]), pack2(e[4], e[5]), pack2(e[6], e[7]));
+                    for (int j = 0; j < CH / 8; ++j) {
+                        float e[8];
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) {
+                            e[i] = fast_exp2(__uint_as_float(sv[j * 8 + i]));
+                            l[ch * CH + j * 8 + i] += e[i];
+                        }
+                        const int cidx = (col0 + ch * CH) / 8 + j;     // 16-byte chunk of the P^T row
+                        *reinterpret_cast<uint4*>(prow + (cidx >> 3) * PANEL + (((cidx & 7) ^ (krow & 7)) << 4)) =
+                            make_uint4(pack2(e[0], e[1]), pack2(e[2], e[3]), pack2(e[4], e[5]), pack2(e[6], e[7]));
+                    }
                 }
             }
             if (!dead) {
@@ -387,65 +517,77 @@ __device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& 
         }
     }
     // ---- end of segment: the accumulator is final once the last PV has completed
-    const uint32_t last = it - 1;
+    const uint32_t last = g - 1;
     wait_u(cx.pv_done + 8 * (last & 1), (last >> 1) & 1);
     tc_fence_after();
-    cx.xch[256 + m * NSLICE + sigma] = l;
+#pragma unroll
+    for (int i = 0; i < NPH; ++i) {
+        float x = l[i];
+#pragma unroll
+        for (int o = 16; o; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+        if (lane == 0) cx.lred[q4 * 128 + col0 + i] = x;
+    }
     soft_sync();
     const int slot = blockIdx.x + sg.s * p.hkv + sg.g;
-    if (owner && warp_on && !dead) {
-        float lt = 0.f;
-#pragma unroll
-        for (int j = 0; j < NSLICE; ++j) lt += cx.xch[256 + m * NSLICE + j];
-        float* wo = p.ws_o + ((size_t)slot * p.mmax + m) * D;
-#pragma unroll
-        for (int cc = 0; cc < D / 32; ++cc) {
-            uint32_t ov[32];
-            tmem_ld32(cx.tm_o + lane_base + cc * 32, ov);
-            tmem_wait_ld();
-            if (row_on) {
-#pragma unroll
-                for (int i = 0; i < 32; i += 4)
-                    *reinterpret_cast<uint4*>(wo + cc * 32 + i) = make_uint4(ov[i], ov[i + 1], ov[i + 2], ov[i + 3]);
-            }
+    if (!dead) {
+        if (tid < M) {
+            const float lt = (cx.lred[tid] + cx.lred[128 + tid]) + (cx.lred[256 + tid] + cx.lred[384 + tid]);
+            const float mn = cx.mneg[tid];
+            *reinterpret_cast<float2*>(p.ws_ml + ((size_t)slot * p.mmax + tid) * 2) = make_float2(mn == UNSET ? -INFINITY : -mn, lt);
         }
-        if (row_on) *reinterpret_cast<float2*>(p.ws_ml + ((size_t)slot * p.mmax + m) * 2) = make_float2(ms, lt);
+        // O^T: lane = head_dim index, column = query row; partials are stored [query row][head_dim]
+        float* wo = p.ws_o + (size_t)slot * p.mmax * D + krow;
+#pragma unroll
+        for (int ch = 0; ch < NCH; ++ch) {
+            uint32_t ov[CH];
+            tmem_ld<CH>(cx.tmem + lane_base + TM_O + col0 + ch * CH, ov);
+            tmem_wait_ld();
+#pragma unroll
+            for (int i = 0; i < CH; ++i)
+                if (col0 + ch * CH + i < M) wo[(size_t)(col0 + ch * CH + i) * D] = __uint_as_float(ov[i]);
+        }
     }
-    soft_sync();                     // the exchange buffer is free again
+    soft_sync();                     // column state and Q^T are free again
     if (!dead) {
         tc_fence_before();
         mbar_arrive(cx.o_free);
     }
 }
 
-template <int D>
 __global__ void __launch_bounds__(THREADS, 1)
 attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
-               const int nk, const int nv)
+               const int nk, const int nv, const int np_max, const int npb)
 {
-    using L = Smem<D>;
     extern __shared__ unsigned char smem_dyn[];
     unsigned char* smem = reinterpret_cast<unsigned char*>(((uintptr_t)smem_dyn + 1023) & ~(uintptr_t)1023);
     Ctx cx;
     cx.nk = nk;
     cx.nv = nv;
+    cx.q_panel = np_max * 128;
+    cx.p_buf = ((np_max + 63) / 64) * PANEL;
+    cx.npb = npb;
     cx.kring = smem;
-    cx.vring = cx.kring + (size_t)nk * L::KV_BYTES;
-    cx.qs = cx.vring + (size_t)nv * L::KV_BYTES;
-    cx.ps = cx.qs + L::Q_BYTES;
-    uint64_t* bars = reinterpret_cast<uint64_t*>(cx.ps + 2 * L::P_BYTES);
+    cx.vring = cx.kring + (size_t)nk * STAGE;
+    cx.ps = cx.vring + (size_t)nv * STAGE;
+    cx.qs = cx.ps + npb * cx.p_buf;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(cx.qs + (D / 64) * cx.q_panel);
     cx.k_full = smem_u32(bars);
-    cx.k_empty = cx.k_full + 8 * MAXRING;
-    cx.v_full = cx.k_empty + 8 * MAXRING;
-    cx.v_empty = cx.v_full + 8 * MAXRING;
-    cx.s_full = cx.v_empty + 8 * MAXRING;
-    cx.p_full = cx.s_full + 8 * NSBUF;
+    cx.k_empty = cx.k_full + 8 * MAXST;
+    cx.v_full = cx.k_empty + 8 * MAXST;
+    cx.v_empty = cx.v_full + 8 * MAXST;
+    cx.v_clean = cx.v_empty + 8 * MAXST;
+    cx.s_full = cx.v_clean + 8 * MAXST;
+    cx.p_full = cx.s_full + 16;
     cx.pv_done = cx.p_full + 16;
     cx.q_ready = cx.pv_done + 16;
     cx.o_free = cx.q_ready + 8;
-    uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bars + 4 * MAXRING + NSBUF + 6);
-    cx.xch = reinterpret_cast<float*>(tmem_holder + 2);      // [256] slice maxima, [256] slice sums
-    cx.pre = reinterpret_cast<int*>(cx.xch + 512);
+    uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bars + 5 * MAXST + 8);
+    cx.mneg = reinterpret_cast<float*>(tmem_holder + 4);
+    cx.alpha = cx.mneg + 128;
+    cx.lred = cx.alpha + 128;
+    cx.cmax = reinterpret_cast<int*>(cx.lred + 512);
+    cx.flags = cx.cmax + 128;
+    cx.pre = cx.flags + 4;
     __shared__ int abort_flag;
     cx.abortp = &abort_flag;
 
@@ -458,14 +600,15 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, con
     const long long hi = cta_first_unit(blockIdx.x + 1, U, p.n_cta);
     if (lo >= hi) return;
     if (threadIdx.x == 0) {
-        for (int i = 0; i < MAXRING; ++i) {
+        for (int i = 0; i < MAXST; ++i) {
             mbar_init(cx.k_full + 8 * i, 1);
             mbar_init(cx.k_empty + 8 * i, 1);
             mbar_init(cx.v_full + 8 * i, 1);
             mbar_init(cx.v_empty + 8 * i, 1);
+            mbar_init(cx.v_clean + 8 * i, 1);
         }
-        for (int i = 0; i < NSBUF; ++i) mbar_init(cx.s_full + 8 * i, 1);
         for (int i = 0; i < 2; ++i) {
+            mbar_init(cx.s_full + 8 * i, 1);
             mbar_init(cx.p_full + 8 * i, NSOFT * 32);
             mbar_init(cx.pv_done + 8 * i, 1);
         }
@@ -483,27 +626,28 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, con
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *reinterpret_cast<volatile uint32_t*>(tmem_holder);
-    cx.tm_s = tmem;
-    cx.tm_o = tmem + NSBUF * TILE;
+    cx.tmem = tmem;
 
     if (warp == W_KPROD) {
-        producer_loop<D>(p, cx, &tm_k, cx.kring, cx.k_full, cx.k_empty, nk, lo, hi, lane);
+        producer_loop(p, cx, &tm_k, cx.kring, cx.k_full, cx.k_empty, nk, lo, hi, lane);
     } else if (warp == W_VPROD) {
-        producer_loop<D>(p, cx, &tm_v, cx.vring, cx.v_full, cx.v_empty, nv, lo, hi, lane);
+        producer_loop(p, cx, &tm_v, cx.vring, cx.v_full, cx.v_empty, nv, lo, hi, lane);
+    } else if (warp == W_VFIX) {
+        vfix_loop(p, cx, lo, hi, lane);
     } else if (warp == W_MMA) {
-        if (lane == 0) mma_loop<D>(p, cx, lo, hi);
+        mma_loop(p, cx, lo, hi, lane);
     } else {
         int s = 0;
-        uint32_t it = 0;
+        uint32_t g = 0;
         long long u = lo;
         bool dead = false;                        // a bounded wait ran out somewhere in the CTA
         while (u < hi) {
             const Segment sg = decode_segment(u, hi, cx.pre, p.hkv, s);
             const int M = p.n_active[sg.s] * p.group;
-            // at most 32 (64) query rows: replicated 4x (2x) along M, 8 (4) threads per row
-            if (M <= 32) softmax_segment<D, 8>(p, cx, sg, it, dead, warp, lane);
-            else if (M <= 64) softmax_segment<D, 16>(p, cx, sg, it, dead, warp, lane);
-            else softmax_segment<D, 32>(p, cx, sg, it, dead, warp, lane);
+            if (M <= 16) softmax_segment<8>(p, cx, sg, g, dead, warp, lane);
+            else if (M <= 32) softmax_segment<16>(p, cx, sg, g, dead, warp, lane);
+            else if (M <= 64) softmax_segment<32>(p, cx, sg, g, dead, warp, lane);
+            else softmax_segment<64>(p, cx, sg, g, dead, warp, lane);
             u = sg.next_u;
         }
     }
@@ -516,19 +660,28 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, con
     }
 }
 
-template <int D>
-int launch_t(const AttnParams& p, cudaStream_t st)
+}  // namespace
+
+namespace fdc {
+
+// bf16, head_dim 128, at most 128 query rows per (scene, KV head); FDC_ERR_SHAPE otherwise (the
+// caller then takes another kernel).
+int launch_attn_tc(const AttnParams& p, int head_dim, cudaStream_t st)
 {
-    using L = Smem<D>;
-    const size_t fixed = 1024 + L::Q_BYTES + 2 * L::P_BYTES + 8 * (4 * MAXRING + NSBUF + 6) + 16 + 2048 + sizeof(int) * (p.batch + 1) + 64;
-    int stages = (int)((227 * 1024 - 256 - fixed) / L::KV_BYTES);
-    if (stages > 2 * MAXRING) stages = 2 * MAXRING;
+    if (head_dim != D || p.mmax > 128) return FDC_ERR_SHAPE;
+    const int np_max = p.mmax <= 16 ? 16 : (p.mmax <= 32 ? 32 : (p.mmax <= 64 ? 64 : 128));
+    const int p_buf = ((np_max + 63) / 64) * PANEL;
+    const int npb = np_max > 64 ? 1 : 2;          // 128 query rows: one P^T buffer, so that four stages still fit
+    const size_t fixed = 1024 + (size_t)npb * p_buf + (size_t)(D / 64) * np_max * 128 + 8 * (5 * MAXST + 8) + 16 +
+                         4 * (128 + 128 + 512 + 128 + 4) + sizeof(int) * (p.batch + 1) + 64;
+    int stages = (int)((227 * 1024 - 256 - fixed) / STAGE);
+    if (stages > 2 * MAXST) stages = 2 * MAXST;
     if (stages < 4) return FDC_ERR_SHAPE;
     const int nk = stages / 2, nv = stages - nk;
-    const size_t smem = fixed + (size_t)stages * L::KV_BYTES;
+    const size_t smem = fixed + (size_t)stages * STAGE;
     static size_t attr_smem = 0;
     if (smem > attr_smem) {
-        cudaError_t e = cudaFuncSetAttribute(attn_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        cudaError_t e = cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return set_cuda_error(e);
         attr_smem = smem;
     }
@@ -537,20 +690,10 @@ int launch_t(const AttnParams& p, cudaStream_t st)
     if (rc) return rc;
     rc = get_kv_tensor_map(p.v, p, D, TILE, &tv);
     if (rc) return rc;
-    attn_tc_kernel<D><<<p.n_cta, THREADS, smem, st>>>(p, tk, tv, nk, nv);
+    attn_tc_kernel<<<p.n_cta, THREADS, smem, st>>>(p, tk, tv, nk, nv, np_max, npb);
     note_launch();
     cudaError_t e = cudaGetLastError();
     return e == cudaSuccess ? FDC_OK : set_cuda_error(e);
-}
-
-}  // namespace
-
-namespace fdc {
-
-// bf16 only, at most 128 query rows per (scene, KV head).
-int launch_attn_tc(const AttnParams& p, int head_dim, cudaStream_t st)
-{
-    return head_dim == 64 ? launch_t<64>(p, st) : launch_t<128>(p, st);
 }
 
 }  // namespace fdc
