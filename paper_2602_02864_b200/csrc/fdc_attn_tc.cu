@@ -12,10 +12,10 @@
 //                      P^T written by the softmax threads (N-major), accumulator in TMEM
 // One persistent CTA per SM:
 //   warps 8, 10  TMA producers: K stages and V stages (128 rows, 128B swizzle) of two rings
-//   warp 9       MMA issuer (one elected thread); allocates / frees TMEM.  S^T is double
+//   warp 9       issues S^T = K Q^T (one elected thread); allocates / frees TMEM.  S^T is double
 //                buffered in TMEM, so K Q^T of round r+1 overlaps the softmax of round r
 //   warp 11      clears the V rows that no branch may see (they can hold anything, NaN included,
-//                and 0 * NaN must not reach the accumulator) and then releases the stage to the MMA
+//                and 0 * NaN must not reach the accumulator), then issues O^T += V^T P^T
 //   warps 0-7    softmax.  Thread = one KV row of the round (TMEM lane) x half of the query
 //                columns.  Eq. 1 is applied by select from the branches' row bitmaps; prefix
 //                tiles skip it.
@@ -37,7 +37,7 @@ constexpr int D = 128;                       // head_dim handled by this kernel
 constexpr int TILE = FDC_TILE_ROWS;          // rows per entry of the visited-tile list
 constexpr int RROWS = 2 * TILE;              // KV rows per round = M of S^T = K of O^T
 constexpr int NSOFT = 8;                     // softmax warps
-constexpr int W_KPROD = 8, W_MMA = 9, W_VPROD = 10, W_VFIX = 11;
+constexpr int W_KPROD = 8, W_QK = 9, W_VPROD = 10, W_PV = 11;
 constexpr int THREADS = 384;
 constexpr uint32_t TMEM_COLS = 512;          // S^T 0 [0,128) | S^T 1 [128,256) | O^T [256,384)
 constexpr uint32_t TM_O = 256;
@@ -152,12 +152,12 @@ __device__ __forceinline__ float ord_to(int i) { return __int_as_float(i ^ ((i >
 
 // Everything a role needs to find its barriers and buffers.
 struct Ctx {
-    uint32_t k_full, k_empty, v_full, v_empty, v_clean, s_full, p_full, pv_done, q_ready, o_free;
+    uint32_t k_full, k_empty, v_full, v_empty, s_full, p_full, pv_done, q_ready, o_free;
     uint32_t tmem;
     unsigned char *kring, *vring, *qs, *ps;
     float *mneg, *alpha, *lred;      // [128] -reference per column, [128] rescale factors, [4][128] partial sums
     int *cmax, *flags;               // [128] column maxima (ordered ints), [2] flags of the raise path
-    int* pre;
+    int *pre, *nact;                 // [batch + 1] tile prefix sums, [batch] active branches per scene
     volatile int* abortp;
     int nk, nv, q_panel, p_buf, npb; // ring depths, bytes per 64-column panel of Q^T, bytes per P^T buffer, P^T buffers (1 or 2)
 };
@@ -214,26 +214,85 @@ __device__ __forceinline__ void producer_loop(const AttnParams& p, const Ctx& cx
     }
 }
 
-// Warp 11: V rows that are invisible to every branch of the scene are cleared in shared memory
-// before the stage is released to O^T += V^T P^T (their P column is exactly 0, but the row may
-// hold NaN or Inf).  Stages wholly inside the prefix are released as they are.
-__device__ __forceinline__ void vfix_loop(const AttnParams& p, const Ctx& cx, long long lo, long long hi, int lane)
+// Warp 9 (one elected thread): S^T[g & 1] = K(stage) Q^T for every round g.  The score buffer is
+// free again once the softmax threads have consumed round g - 2, which they signal with p_full.
+__device__ __forceinline__ void qk_loop(const AttnParams& p, const Ctx& cx, long long lo, long long hi, int lane)
 {
+    const uint64_t q_desc = smem_desc(smem_u32(cx.qs), 16, 1024);
+    const uint64_t k_desc0 = smem_desc(smem_u32(cx.kring), 16, 1024);
+    const uint64_t qp16 = (uint64_t)(cx.q_panel >> 4);
     int s = 0;
-    uint32_t g = 0;
+    uint32_t g = 0, seg = 0;
+    int st = 0;
+    uint32_t kph = 0;                               // ring position and phase of the K stage of round g
     long long u = lo;
     int ok = 1;
     while (u < hi && ok) {
         const Segment sg = decode_segment(u, hi, cx.pre, p.hkv, s);
-        const int A = p.n_active[sg.s];
+        const int nr = (sg.j1 - sg.j0 + 1) >> 1;
+        if (lane == 0) {
+            const int M = cx.nact[sg.s] * p.group;
+            const int NP = M <= 16 ? 16 : (M <= 32 ? 32 : (M <= 64 ? 64 : 128));
+            const uint32_t idesc_qk = instr_desc(RROWS, NP, 0);
+            bool good = mbar_wait(cx.q_ready, seg & 1, cx.abortp, p.status);
+            for (int t = 0; t < nr && good; ++t, ++g) {
+                good = mbar_wait(cx.k_full + 8 * st, kph, cx.abortp, p.status);
+                if (good && g >= 2) good = mbar_wait(cx.p_full + 8 * (g & 1), ((g - 2) >> 1) & 1, cx.abortp, p.status);
+                if (!good) break;
+                tc_fence_after();
+                const uint64_t kd = k_desc0 + (uint64_t)((st * STAGE) >> 4);
+                const uint32_t d = cx.tmem + (g & 1) * 128;
+#pragma unroll
+                for (int ks = 0; ks < D / 16; ++ks)
+                    umma(d, kd + (uint64_t)(((ks >> 2) * PANEL + (ks & 3) * 32) >> 4), q_desc + (ks >> 2) * qp16 + (uint64_t)(((ks & 3) * 32) >> 4),
+                         idesc_qk, ks > 0);
+                umma_commit(cx.k_empty + 8 * st);
+                umma_commit(cx.s_full + 8 * (g & 1));
+                if (++st == cx.nk) {
+                    st = 0;
+                    kph ^= 1;
+                }
+            }
+            ok = good;
+        }
+        ok = __shfl_sync(0xffffffffu, ok, 0);
+        g = __shfl_sync(0xffffffffu, g, 0);
+        st = __shfl_sync(0xffffffffu, st, 0);
+        kph = __shfl_sync(0xffffffffu, kph, 0);
+        ++seg;
+        u = sg.next_u;
+    }
+}
+
+// Warp 11: O^T += V^T(stage) P^T[g & 1] for every round g (one elected thread issues).  Before
+// that the whole warp clears the V rows of the stage that are invisible to every branch of the
+// scene: their P^T row is exactly 0, but the rows can hold anything (NaN, Inf) and 0 * NaN must
+// not reach the accumulator.  Stages wholly inside the prefix need no such pass.
+__device__ __forceinline__ void pv_loop(const AttnParams& p, const Ctx& cx, long long lo, long long hi, int lane)
+{
+    const uint64_t v_desc0 = smem_desc(smem_u32(cx.vring), PANEL, 1024);
+    const uint64_t p_desc0 = smem_desc(smem_u32(cx.ps), PANEL, 1024);
+    const uint32_t tm_o = cx.tmem + TM_O;
+    int s = 0;
+    uint32_t g = 0, seg = 0;
+    int st = 0;
+    uint32_t vph = 0;
+    long long u = lo;
+    int ok = 1;
+    while (u < hi && ok) {
+        const Segment sg = decode_segment(u, hi, cx.pre, p.hkv, s);
+        const int A = cx.nact[sg.s];
+        const int M = A * p.group;
+        const int NP = M <= 16 ? 16 : (M <= 32 ? 32 : (M <= 64 ? 64 : 128));
+        const uint32_t idesc_pv = instr_desc(D, NP, 1);
+        int t = 0;
         for (int jb = sg.j0; jb < sg.j1 && ok; jb += 32) {
             const int jn = sg.j1 - jb < 32 ? sg.j1 - jb : 32;
             const int my_tile = lane < jn ? p.tiles[(size_t)sg.s * p.ntile_max + jb + lane] : 0;
-            for (int k = 0; k < jn && ok; k += 2, ++g) {
+            for (int k = 0; k < jn && ok; k += 2, ++g, ++t) {
                 const int nt = jn - k < 2 ? 1 : 2;
-                const int st = g % cx.nv;
                 int okw = 1;
-                if (lane == 0) okw = mbar_wait(cx.v_full + 8 * st, (g / cx.nv) & 1, cx.abortp, p.status);
+                if (lane == 0) okw = mbar_wait(cx.v_full + 8 * st, vph, cx.abortp, p.status);
                 ok = __shfl_sync(0xffffffffu, okw, 0);
                 if (!ok) break;
                 unsigned char* vs = cx.vring + (size_t)st * STAGE;
@@ -246,91 +305,55 @@ __device__ __forceinline__ void vfix_loop(const AttnParams& p, const Ctx& cx, lo
                         um |= tile_rowmask(p.mask + ((size_t)sg.s * p.max_active + b) * p.W, p.W, p.P, tile);
                     const uint32_t ul = __reduce_or_sync(0xffffffffu, (uint32_t)um);
                     const uint32_t uh = __reduce_or_sync(0xffffffffu, (uint32_t)(um >> 32));
-                    uint64_t z = ~(((uint64_t)uh << 32) | ul);
-                    // two rows per step: lanes 0-15 clear one row (2 panels x 8 chunks of 16 bytes), lanes 16-31 the next
-                    while (z) {
-                        const int r0 = __ffsll((long long)z) - 1;
-                        z &= z - 1;
-                        int r1 = -1;
-                        if (z) {
-                            r1 = __ffsll((long long)z) - 1;
-                            z &= z - 1;
-                        }
-                        const int r = lane < 16 ? r0 : r1;
-                        if (r >= 0) {
-                            const int l16 = lane & 15;
-                            *reinterpret_cast<uint4*>(vs + (l16 >> 3) * PANEL + (i * TILE + r) * 128 + ((l16 & 7) << 4)) =
-                                make_uint4(0u, 0u, 0u, 0u);
+                    const uint64_t z = ~(((uint64_t)uh << 32) | ul);
+                    if (z) {
+                        // lane l clears rows l and l + 32 of the tile if nobody sees them (2 panels x 8 chunks of 16 bytes)
+#pragma unroll
+                        for (int hr = 0; hr < 2; ++hr) {
+                            const int r = lane + 32 * hr;
+                            if ((z >> r) & 1) {
+                                unsigned char* row = vs + (i * TILE + r) * 128;
+#pragma unroll
+                                for (int ch = 0; ch < 8; ++ch) {
+                                    // rotate the chunk order by the row so that the lanes of a warp hit different banks
+                                    const int cc = ((ch + r) & 7) << 4;
+                                    *reinterpret_cast<uint4*>(row + cc) = make_uint4(0u, 0u, 0u, 0u);
+                                    *reinterpret_cast<uint4*>(row + PANEL + cc) = make_uint4(0u, 0u, 0u, 0u);
+                                }
+                            }
                         }
                         touched = true;
                     }
                 }
                 if (touched) fence_async_smem();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(cx.v_clean + 8 * st);
-            }
-        }
-        u = sg.next_u;
-    }
-}
-
-// The MMA issuer (whole warp follows the loop, lane 0 waits and issues).
-__device__ __forceinline__ void mma_loop(const AttnParams& p, const Ctx& cx, long long lo, long long hi, int lane)
-{
-    const uint64_t q_desc = smem_desc(smem_u32(cx.qs), 16, 1024);
-    const uint64_t k_desc0 = smem_desc(smem_u32(cx.kring), 16, 1024);
-    const uint64_t v_desc0 = smem_desc(smem_u32(cx.vring), PANEL, 1024);
-    const uint64_t p_desc0 = smem_desc(smem_u32(cx.ps), PANEL, 1024);
-    const uint32_t tm_o = cx.tmem + TM_O;
-    int s = 0;
-    uint32_t g0 = 0, seg = 0;
-    long long u = lo;
-    int ok = 1;
-    while (u < hi && ok) {
-        const Segment sg = decode_segment(u, hi, cx.pre, p.hkv, s);
-        const int ntile = sg.j1 - sg.j0;
-        const int nr = (ntile + 1) >> 1;
-        if (lane == 0) {
-            int M = p.n_active[sg.s] * p.group;
-            const int NP = M <= 16 ? 16 : (M <= 32 ? 32 : (M <= 64 ? 64 : 128));
-            const uint32_t idesc_qk = instr_desc(RROWS, NP, 0), idesc_pv = instr_desc(D, NP, 1);
-            // S^T[g & 1] = K(stage) Q^T
-            auto issue_qk = [&](uint32_t g) -> bool {
-                const int st = g % cx.nk;
-                if (!mbar_wait(cx.k_full + 8 * st, (g / cx.nk) & 1, cx.abortp, p.status)) return false;
-                tc_fence_after();
-                const uint64_t kd = k_desc0 + (uint64_t)((st * STAGE) >> 4);
+                if (lane == 0) {
+                    bool good = mbar_wait(cx.p_full + 8 * (g & 1), (g >> 1) & 1, cx.abortp, p.status);
+                    if (good && t == 0 && seg > 0) good = mbar_wait(cx.o_free, (seg - 1) & 1, cx.abortp, p.status);
+                    if (good) {
+                        tc_fence_after();
+                        const uint64_t vd = v_desc0 + (uint64_t)((st * STAGE) >> 4);
+                        const uint64_t pd = p_desc0 + (uint64_t)((((g & 1) & (cx.npb - 1)) * cx.p_buf) >> 4);
 #pragma unroll
-                for (int ks = 0; ks < D / 16; ++ks)
-                    umma(cx.tmem + (g & 1) * 128, kd + (uint64_t)(((ks >> 2) * PANEL + (ks & 3) * 32) >> 4),
-                         q_desc + (uint64_t)(((ks >> 2) * cx.q_panel + (ks & 3) * 32) >> 4), idesc_qk, ks > 0);
-                umma_commit(cx.k_empty + 8 * st);
-                umma_commit(cx.s_full + 8 * (g & 1));
-                return true;
-            };
-            bool good = mbar_wait(cx.q_ready, seg & 1, cx.abortp, p.status);
-            for (int a = 0; a < 2 && a < nr && good; ++a) good = issue_qk(g0 + a);
-            for (int t = 0; t < nr && good; ++t) {
-                const uint32_t g = g0 + t;
-                const int rows = (t == nr - 1 && (ntile & 1)) ? TILE : RROWS;
-                good = mbar_wait(cx.p_full + 8 * (g & 1), (g >> 1) & 1, cx.abortp, p.status);
-                if (good && t == 0 && seg > 0) good = mbar_wait(cx.o_free, (seg - 1) & 1, cx.abortp, p.status);
-                const int st = g % cx.nv;
-                if (good) good = mbar_wait(cx.v_clean + 8 * st, (g / cx.nv) & 1, cx.abortp, p.status);
-                if (!good) break;
-                tc_fence_after();
-                const uint64_t vd = v_desc0 + (uint64_t)((st * STAGE) >> 4);
-                const uint64_t pd = p_desc0 + (uint64_t)((((g & 1) & (cx.npb - 1)) * cx.p_buf) >> 4);
-                for (int kk = 0; kk < rows / 16; ++kk)
-                    umma(tm_o, vd + (uint64_t)((kk * 2048) >> 4), pd + (uint64_t)((kk * 2048) >> 4), idesc_pv, (t > 0 || kk > 0) ? 1u : 0u);
-                umma_commit(cx.v_empty + 8 * st);
-                umma_commit(cx.pv_done + 8 * (g & 1));
-                if (t + 2 < nr) good = issue_qk(g + 2);
+                        for (int kk = 0; kk < 4; ++kk)
+                            umma(tm_o, vd + (uint64_t)((kk * 2048) >> 4), pd + (uint64_t)((kk * 2048) >> 4), idesc_pv, (t > 0 || kk > 0) ? 1u : 0u);
+                        if (nt == 2) {                                       // a one-tile round has 64 KV rows
+#pragma unroll
+                            for (int kk = 4; kk < 8; ++kk)
+                                umma(tm_o, vd + (uint64_t)((kk * 2048) >> 4), pd + (uint64_t)((kk * 2048) >> 4), idesc_pv, 1u);
+                        }
+                        umma_commit(cx.v_empty + 8 * st);
+                        umma_commit(cx.pv_done + 8 * (g & 1));
+                    }
+                    okw = good;
+                }
+                ok = __shfl_sync(0xffffffffu, okw, 0);
+                if (++st == cx.nv) {
+                    st = 0;
+                    vph ^= 1;
+                }
             }
-            ok = good;
         }
-        ok = __shfl_sync(0xffffffffu, ok, 0);
-        g0 += nr;
         ++seg;
         u = sg.next_u;
     }
@@ -350,7 +373,7 @@ __device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& 
     const uint32_t lane_base = (uint32_t)(q4 * 32) << 16;
     const int col0 = half * NPH;
     const float c = p.scale_log2;
-    const int A = p.n_active[sg.s];
+    const int A = cx.nact[sg.s];
     const int M = A * p.group;
     const int G = p.group;
     auto wait_u = [&](uint32_t bar, uint32_t parity) {    // warp-uniform outcome
@@ -380,6 +403,12 @@ __device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& 
     float l[NPH];
 #pragma unroll
     for (int i = 0; i < NPH; ++i) l[i] = 0.f;
+    // -reference of this thread's columns: in registers when they fit, else read from shared memory
+    constexpr bool REF_REGS = NPH <= 32;
+    float mr[REF_REGS ? NPH : 1];
+#pragma unroll
+    for (int i = 0; i < (REF_REGS ? NPH : 1); ++i) mr[i] = UNSET;
+#define FDC_MNEG(i) (REF_REGS ? mr[REF_REGS ? (i) : 0] : cx.mneg[col0 + (i)])
 
     const int ntile = sg.j1 - sg.j0;
     int t = 0;                                    // round within the segment
@@ -393,45 +422,42 @@ __device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& 
             const int tile = __shfl_sync(0xffffffffu, my_tile, (k + ti) & 31);
             const bool live = ti < nt && !dead;                       // rows 64..127 of a one-tile round hold nothing
             const bool masked = live && tile * TILE + TILE > p.P;
-            // visibility of this warp's 32 rows for branch `lane` (and `lane + 32`), Eq. 1
-            uint32_t wlo = 0xffffffffu, whi = 0xffffffffu;
+            // Eq. 1 for this thread's KV row: bit i of vis <=> column col0 + i may see the row
+            uint64_t vis = ~0ull;
             if (masked) {
                 uint64_t m0 = 0ull, m1 = 0ull;
                 if (lane < A) m0 = tile_rowmask(p.mask + ((size_t)sg.s * p.max_active + lane) * p.W, p.W, p.P, tile);
                 if (lane + 32 < A) m1 = tile_rowmask(p.mask + ((size_t)sg.s * p.max_active + lane + 32) * p.W, p.W, p.P, tile);
-                wlo = (q4 & 1) ? (uint32_t)(m0 >> 32) : (uint32_t)m0;
-                whi = (q4 & 1) ? (uint32_t)(m1 >> 32) : (uint32_t)m1;
+                // rows of this warp for branch `lane` / `lane + 32`
+                const uint32_t wlo = (q4 & 1) ? (uint32_t)(m0 >> 32) : (uint32_t)m0;
+                const uint32_t whi = (q4 & 1) ? (uint32_t)(m1 >> 32) : (uint32_t)m1;
+                vis = 0ull;
+                const int b_lo = col0 / G, b_hi = (col0 + NPH - 1) / G;
+                for (int bq = b_lo; bq <= b_hi; ++bq) {
+                    const uint32_t bits = __shfl_sync(0xffffffffu, bq < 32 ? wlo : whi, bq & 31);
+                    if ((bits >> lane) & 1) {
+                        const int c_lo = bq * G - col0 < 0 ? 0 : bq * G - col0;
+                        const int c_hi = (bq + 1) * G - col0 > NPH ? NPH : (bq + 1) * G - col0;     // exclusive
+                        const uint64_t span = c_hi - c_lo == 64 ? ~0ull : ((1ull << (c_hi - c_lo)) - 1ull);
+                        vis |= span << c_lo;
+                    }
+                }
             }
             wait_u(cx.s_full + 8 * b, (g >> 1) & 1);
             tc_fence_after();
             const uint32_t s_addr = cx.tmem + lane_base + b * 128 + col0;
-            // args[i] = score * scale * log2(e) - reference, -inf where Eq. 1 hides the row
-            auto load_args = [&](int chunk, uint32_t (&sv)[CH], bool minus_ref) {
-                tmem_ld<CH>(s_addr + chunk * CH, sv);
-                tmem_wait_ld();
-                int bq = (col0 + chunk * CH) / G, rem = (col0 + chunk * CH) - bq * G;
-#pragma unroll
-                for (int i = 0; i < CH; ++i) {
-                    float a = minus_ref ? fmaf(__uint_as_float(sv[i]), c, cx.mneg[col0 + chunk * CH + i]) : __uint_as_float(sv[i]) * c;
-                    if (masked) {
-                        const uint32_t bits = __shfl_sync(0xffffffffu, bq < 32 ? wlo : whi, bq & 31);
-                        if (!((bits >> lane) & 1)) a = -INFINITY;
-                        if (++rem == G) {
-                            rem = 0;
-                            ++bq;
-                        }
-                    }
-                    sv[i] = __float_as_uint(a);
-                }
-            };
-            uint32_t sv[CH];
-            float amax = -INFINITY;
+            uint32_t sv[CH];                       // raw scores of the current chunk (-inf where hidden)
+            float amax = -INFINITY;                // max over this thread's columns of score * c - reference
             if (live) {
 #pragma unroll
                 for (int ch = 0; ch < NCH; ++ch) {
-                    load_args(ch, sv, true);
+                    tmem_ld<CH>(s_addr + ch * CH, sv);
+                    tmem_wait_ld();
 #pragma unroll
-                    for (int i = 0; i < CH; ++i) amax = fmaxf(amax, __uint_as_float(sv[i]));
+                    for (int i = 0; i < CH; ++i) {
+                        if (masked && !((vis >> (ch * CH + i)) & 1)) sv[i] = 0xff800000u;
+                        amax = fmaxf(amax, fmaf(__uint_as_float(sv[i]), c, FDC_MNEG(ch * CH + i)));
+                    }
                 }
             }
             // does some column need a (higher) reference?  first visible score, or a jump of more than 2^8
@@ -439,10 +465,15 @@ __device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& 
                 if (live) {
 #pragma unroll
                     for (int ch = 0; ch < NCH; ++ch) {
-                        load_args(ch, sv, false);
+                        if (NCH > 1) {
+                            tmem_ld<CH>(s_addr + ch * CH, sv);
+                            tmem_wait_ld();
+                        }
 #pragma unroll
                         for (int i = 0; i < CH; ++i) {
-                            const int wm = __reduce_max_sync(0xffffffffu, ord_of(__uint_as_float(sv[i])));
+                            float x = __uint_as_float(sv[i]) * c;
+                            if (NCH > 1 && masked && !((vis >> (ch * CH + i)) & 1)) x = -INFINITY;
+                            const int wm = __reduce_max_sync(0xffffffffu, ord_of(x));
                             if (lane == 0) atomicMax(&cx.cmax[col0 + ch * CH + i], wm);
                         }
                     }
@@ -450,20 +481,22 @@ __device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& 
                 if (tid == 0) cx.flags[0] = 0;
                 soft_sync();
                 if (tid < NP) {
-                    const float mr = ord_to(cx.cmax[tid]);
+                    const float mx = ord_to(cx.cmax[tid]);
                     const float old = cx.mneg[tid];                    // -reference, or UNSET
                     float al = 1.f;
                     if (old == UNSET) {
-                        if (mr != -INFINITY) cx.mneg[tid] = -mr;
-                    } else if (mr > RAISE_LOG2 - old) {
-                        al = fast_exp2(-old - mr);
-                        cx.mneg[tid] = -mr;
+                        if (mx != -INFINITY) cx.mneg[tid] = -mx;
+                    } else if (mx > RAISE_LOG2 - old) {
+                        al = fast_exp2(-old - mx);
+                        cx.mneg[tid] = -mx;
                         cx.flags[0] = 1;
                     }
                     cx.alpha[tid] = al;
                     cx.cmax[tid] = INT_MIN;
                 }
                 soft_sync();
+#pragma unroll
+                for (int i = 0; i < (REF_REGS ? NPH : 1); ++i) mr[i] = cx.mneg[col0 + i];
                 if (cx.flags[0]) {                                     // a reference moved: rescale sums and accumulator
 #pragma unroll
                     for (int i = 0; i < NPH; ++i) l[i] *= cx.alpha[col0 + i];
@@ -484,7 +517,6 @@ __device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& 
                         }
                     }
                 }
-                if (NCH == 1 && live) load_args(0, sv, true);
             }
             // the P^T buffer is still being read until the PV that used it last (two rounds ago, or
             // the previous round when there is a single buffer) has completed
@@ -494,13 +526,19 @@ __device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& 
                 unsigned char* prow = cx.ps + (b & (cx.npb - 1)) * cx.p_buf + krow * 128;
 #pragma unroll
                 for (int ch = 0; ch < NCH; ++ch) {
-                    if (NCH > 1) load_args(ch, sv, true);
+                    if (NCH > 1) {
+                        tmem_ld<CH>(s_addr + ch * CH, sv);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int i = 0; i < CH; ++i)
+                            if (masked && !((vis >> (ch * CH + i)) & 1)) sv[i] = 0xff800000u;
+                    }
 #pragma unroll
                     for (int j = 0; j < CH / 8; ++j) {
                         float e[8];
 #pragma unroll
                         for (int i = 0; i < 8; ++i) {
-                            e[i] = fast_exp2(__uint_as_float(sv[j * 8 + i]));
+                            e[i] = fast_exp2(fmaf(__uint_as_float(sv[j * 8 + i]), c, FDC_MNEG(ch * CH + j * 8 + i)));
                             l[ch * CH + j * 8 + i] += e[i];
                         }
                         const int cidx = (col0 + ch * CH) / 8 + j;     // 16-byte chunk of the P^T row
@@ -516,6 +554,7 @@ __device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& 
             }
         }
     }
+#undef FDC_MNEG
     // ---- end of segment: the accumulator is final once the last PV has completed
     const uint32_t last = g - 1;
     wait_u(cx.pv_done + 8 * (last & 1), (last >> 1) & 1);
@@ -575,24 +614,25 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, con
     cx.k_empty = cx.k_full + 8 * MAXST;
     cx.v_full = cx.k_empty + 8 * MAXST;
     cx.v_empty = cx.v_full + 8 * MAXST;
-    cx.v_clean = cx.v_empty + 8 * MAXST;
-    cx.s_full = cx.v_clean + 8 * MAXST;
+    cx.s_full = cx.v_empty + 8 * MAXST;
     cx.p_full = cx.s_full + 16;
     cx.pv_done = cx.p_full + 16;
     cx.q_ready = cx.pv_done + 16;
     cx.o_free = cx.q_ready + 8;
-    uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bars + 5 * MAXST + 8);
+    uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bars + 4 * MAXST + 8);
     cx.mneg = reinterpret_cast<float*>(tmem_holder + 4);
     cx.alpha = cx.mneg + 128;
     cx.lred = cx.alpha + 128;
     cx.cmax = reinterpret_cast<int*>(cx.lred + 512);
     cx.flags = cx.cmax + 128;
     cx.pre = cx.flags + 4;
+    cx.nact = cx.pre + p.batch + 1;
     __shared__ int abort_flag;
     cx.abortp = &abort_flag;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 0) abort_flag = 0;
+    for (int i = threadIdx.x; i < p.batch; i += THREADS) cx.nact[i] = p.n_active[i];
     const long long total = scan_ntiles(p.ntiles, p.batch, cx.pre);
     const long long U = total * p.hkv;
     if (U == 0) return;
@@ -605,7 +645,6 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, con
             mbar_init(cx.k_empty + 8 * i, 1);
             mbar_init(cx.v_full + 8 * i, 1);
             mbar_init(cx.v_empty + 8 * i, 1);
-            mbar_init(cx.v_clean + 8 * i, 1);
         }
         for (int i = 0; i < 2; ++i) {
             mbar_init(cx.s_full + 8 * i, 1);
@@ -617,7 +656,7 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, con
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         fence_async_smem();
     }
-    if (warp == W_MMA) {
+    if (warp == W_QK) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_holder)), "r"(TMEM_COLS)
                      : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -632,10 +671,10 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, con
         producer_loop(p, cx, &tm_k, cx.kring, cx.k_full, cx.k_empty, nk, lo, hi, lane);
     } else if (warp == W_VPROD) {
         producer_loop(p, cx, &tm_v, cx.vring, cx.v_full, cx.v_empty, nv, lo, hi, lane);
-    } else if (warp == W_VFIX) {
-        vfix_loop(p, cx, lo, hi, lane);
-    } else if (warp == W_MMA) {
-        mma_loop(p, cx, lo, hi, lane);
+    } else if (warp == W_PV) {
+        pv_loop(p, cx, lo, hi, lane);
+    } else if (warp == W_QK) {
+        qk_loop(p, cx, lo, hi, lane);
     } else {
         int s = 0;
         uint32_t g = 0;
@@ -643,7 +682,7 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, con
         bool dead = false;                        // a bounded wait ran out somewhere in the CTA
         while (u < hi) {
             const Segment sg = decode_segment(u, hi, cx.pre, p.hkv, s);
-            const int M = p.n_active[sg.s] * p.group;
+            const int M = cx.nact[sg.s] * p.group;
             if (M <= 16) softmax_segment<8>(p, cx, sg, g, dead, warp, lane);
             else if (M <= 32) softmax_segment<16>(p, cx, sg, g, dead, warp, lane);
             else if (M <= 64) softmax_segment<32>(p, cx, sg, g, dead, warp, lane);
@@ -654,7 +693,7 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, con
     // ---- teardown: everybody is done with TMEM before it is freed
     tc_fence_before();
     __syncthreads();
-    if (warp == W_MMA) {
+    if (warp == W_QK) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(TMEM_COLS) : "memory");
     }
@@ -672,8 +711,8 @@ int launch_attn_tc(const AttnParams& p, int head_dim, cudaStream_t st)
     const int np_max = p.mmax <= 16 ? 16 : (p.mmax <= 32 ? 32 : (p.mmax <= 64 ? 64 : 128));
     const int p_buf = ((np_max + 63) / 64) * PANEL;
     const int npb = np_max > 64 ? 1 : 2;          // 128 query rows: one P^T buffer, so that four stages still fit
-    const size_t fixed = 1024 + (size_t)npb * p_buf + (size_t)(D / 64) * np_max * 128 + 8 * (5 * MAXST + 8) + 16 +
-                         4 * (128 + 128 + 512 + 128 + 4) + sizeof(int) * (p.batch + 1) + 64;
+    const size_t fixed = 1024 + (size_t)npb * p_buf + (size_t)(D / 64) * np_max * 128 + 8 * (4 * MAXST + 8) + 16 +
+                         4 * (128 + 128 + 512 + 128 + 4) + sizeof(int) * (2 * p.batch + 1) + 64;
     int stages = (int)((227 * 1024 - 256 - fixed) / STAGE);
     if (stages > 2 * MAXST) stages = 2 * MAXST;
     if (stages < 4) return FDC_ERR_SHAPE;
