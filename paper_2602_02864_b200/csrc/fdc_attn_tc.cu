@@ -20,8 +20,9 @@
 //                columns.  Eq. 1 is applied by select from the branches' row bitmaps; prefix
 //                tiles skip it.
 // The softmax reference of a query column is raised lazily: it is set from the column maximum
-// of the first round and raised again only when some score exceeds it by more than 2^8 (one
-// barrier-wide OR per round detects that).  Sum and accumulator use the same reference, so the
+// of the first round (a column that sees no row yet borrows the round's highest maximum) and
+// raised again only when some score exceeds it by more than 2^16 (one barrier-wide OR per round
+// detects that).  Sum and accumulator use the same reference, so the
 // result is exact; the column sums are kept per thread and reduced at the end of a segment.
 #include <cudaTypedefs.h>
 
@@ -44,7 +45,7 @@ constexpr uint32_t TM_O = 256;
 constexpr int PANEL = RROWS * 128;           // 128 rows x 128 bytes (64 bf16 columns)
 constexpr int STAGE = (D / 64) * PANEL;      // one K (or V) stage: 128 rows x head_dim
 constexpr int MAXST = 4;                     // stages per ring at most
-constexpr float RAISE_LOG2 = 8.f;
+constexpr float RAISE_LOG2 = 16.f;
 constexpr float UNSET = 1.0e30f;             // -reference of a column that has seen nothing yet
 
 // ---------------------------------------------------------------- tcgen05 wrappers
@@ -359,6 +360,112 @@ __device__ __forceinline__ void pv_loop(const AttnParams& p, const Ctx& cx, long
     }
 }
 
+// The rare path of the softmax, kept out of line so that the per-round loop stays small: some
+// score exceeded its column's reference by more than 2^16 (or a column saw its first score).
+// Column maxima of the round are gathered (warp max, one shared-memory slot per warp), references
+// that are unset or too low are replaced, alpha[n] = 2^(old - new) is published, and the
+// accumulator O^T is rescaled when it already holds something.  Called by all softmax threads.
+// Returns bit 0: some reference moved (the caller rescales its partial sums by alpha),
+// bit 1: a bounded wait ran out.
+struct RaiseArgs {
+    float* mneg;                 // column state in shared memory: mneg[128], alpha[128], lred[512], cmax[128], flags[4]
+    volatile int* abortp;
+    int32_t* status;
+    uint32_t s_addr, o_addr;     // TMEM addresses of this thread's first score / accumulator column
+    uint32_t pv_bar, pv_parity;  // completion of the previous round's O^T += V^T P^T
+    uint64_t vis;                // Eq. 1 bits of this thread's columns
+    float c;
+    int col0, live, rescale_o, dead;
+};
+template <int NPH>
+__device__ __noinline__ int raise_references(const RaiseArgs a)
+{
+    constexpr int NP = 2 * NPH;
+    constexpr int CH = NPH < 32 ? NPH : 32;
+    constexpr int NCH = NPH / CH;
+    float* alpha = a.mneg + 128;
+    int* wmax = reinterpret_cast<int*>(a.mneg + 256);      // [4][128]: maxima per row quadrant (shares the lred block)
+    int* flags = reinterpret_cast<int*>(a.mneg + 768) + 128;
+    const int tid = threadIdx.x, lane = threadIdx.x & 31, q4 = (threadIdx.x >> 5) & 3;
+    bool dead = a.dead != 0;
+#pragma unroll
+    for (int ch = 0; ch < NCH; ++ch) {
+        float mine = -INFINITY;                              // lane i ends up with the maximum of column ch * CH + i
+        if (a.live) {
+            uint32_t sv[CH];
+            tmem_ld<CH>(a.s_addr + ch * CH, sv);
+            tmem_wait_ld();
+            float v[CH];
+#pragma unroll
+            for (int i = 0; i < CH; ++i) v[i] = ((a.vis >> (ch * CH + i)) & 1) ? __uint_as_float(sv[i]) * a.c : -INFINITY;
+            // lanes whose index differs in bits >= CH hold rows of the same columns: plain max
+#pragma unroll
+            for (int o = 16; o >= CH; o >>= 1)
+#pragma unroll
+                for (int i = 0; i < CH; ++i) v[i] = fmaxf(v[i], __shfl_xor_sync(0xffffffffu, v[i], o));
+            // transpose-reduce: at distance k a lane keeps the half of the columns that matches its bit k
+#pragma unroll
+            for (int k = CH / 2; k >= 1; k >>= 1) {
+                const bool up = (lane & k) != 0;
+#pragma unroll
+                for (int i = 0; i < k; ++i) {
+                    const float recv = __shfl_xor_sync(0xffffffffu, up ? v[i] : v[i + k], k);
+                    v[i] = fmaxf(up ? v[i + k] : v[i], recv);
+                }
+            }
+            mine = v[0];
+        }
+        if (lane < CH) wmax[q4 * 128 + a.col0 + ch * CH + lane] = ord_of(mine);
+    }
+    if (tid == 0) flags[0] = 0;
+    soft_sync();
+    if (tid < ((NP + 31) & ~31)) {                         // whole warps (the shuffles below need all lanes)
+        // highest column maximum of the round (every warp of these threads computes it for itself)
+        int gm = INT_MIN;
+        for (int n = lane; n < NP; n += 32)
+            gm = max(gm, max(max(wmax[n], wmax[128 + n]), max(wmax[256 + n], wmax[384 + n])));
+#pragma unroll
+        for (int o = 16; o; o >>= 1) gm = max(gm, __shfl_xor_sync(0xffffffffu, gm, o));
+        if (tid < NP) {
+            const int m01 = max(wmax[tid], wmax[128 + tid]), m23 = max(wmax[256 + tid], wmax[384 + tid]);
+            const float mx = ord_to(max(m01, m23));
+            const float old = a.mneg[tid];                     // -reference, or UNSET
+            float al = 1.f;
+            if (old == UNSET) {
+                // a column that sees no row yet borrows the round's highest reference: it will rarely have
+                // to be raised later, and lower scores only make its terms smaller (far from underflow)
+                const float ref = mx != -INFINITY ? mx : ord_to(gm);
+                if (ref != -INFINITY) a.mneg[tid] = -ref;
+            } else if (mx > RAISE_LOG2 - old) {
+                al = fast_exp2(-old - mx);
+                a.mneg[tid] = -mx;
+                flags[0] = 1;
+            }
+            alpha[tid] = al;
+        }
+    }
+    soft_sync();
+    const int moved = flags[0];
+    if (moved && a.rescale_o) {
+        if (!dead && !mbar_wait(a.pv_bar, a.pv_parity, a.abortp, a.status)) dead = true;   // no MMA may be writing O^T
+        dead = __any_sync(0xffffffffu, dead);
+        tc_fence_after();
+        if (!dead) {
+#pragma unroll
+            for (int ch = 0; ch < NCH; ++ch) {
+                uint32_t ov[CH];
+                tmem_ld<CH>(a.o_addr + ch * CH, ov);
+                tmem_wait_ld();
+#pragma unroll
+                for (int i = 0; i < CH; ++i) ov[i] = __float_as_uint(__uint_as_float(ov[i]) * alpha[a.col0 + ch * CH + i]);
+                tmem_st<CH>(a.o_addr + ch * CH, ov);
+            }
+            tmem_wait_st();
+        }
+    }
+    return moved | (dead ? 2 : 0);
+}
+
 // The softmax warps' work on one segment; NPH = query columns per thread (half of NP).
 template <int NPH>
 __device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& cx, const Segment& sg, uint32_t& g, bool& dead,
@@ -392,12 +499,10 @@ __device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& 
             }
             *reinterpret_cast<uint4*>(cx.qs + (ch >> 3) * cx.q_panel + n * 128 + (((ch & 7) ^ (n & 7)) << 4)) = v;
         }
-        if (tid < NP) {
-            cx.mneg[tid] = UNSET;
-            cx.cmax[tid] = INT_MIN;
-        }
+        if (tid < NP) cx.mneg[tid] = UNSET;
         fence_async_smem();
-        if (!dead) mbar_arrive(cx.q_ready);
+        __syncwarp();
+        if (!dead && lane == 0) mbar_arrive(cx.q_ready);
         soft_sync();
     }
     float l[NPH];
@@ -453,69 +558,39 @@ __device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& 
                 for (int ch = 0; ch < NCH; ++ch) {
                     tmem_ld<CH>(s_addr + ch * CH, sv);
                     tmem_wait_ld();
+                    if (masked) {                                      // uniform branch: prefix rounds skip the selects
+                        const uint32_t vb = (uint32_t)(vis >> (ch * CH));
 #pragma unroll
-                    for (int i = 0; i < CH; ++i) {
-                        if (masked && !((vis >> (ch * CH + i)) & 1)) sv[i] = 0xff800000u;
-                        amax = fmaxf(amax, fmaf(__uint_as_float(sv[i]), c, FDC_MNEG(ch * CH + i)));
+                        for (int i = 0; i < CH; ++i)
+                            if (!((vb >> i) & 1)) sv[i] = 0xff800000u;
                     }
+#pragma unroll
+                    for (int i = 0; i < CH; ++i) amax = fmaxf(amax, fmaf(__uint_as_float(sv[i]), c, FDC_MNEG(ch * CH + i)));
                 }
             }
-            // does some column need a (higher) reference?  first visible score, or a jump of more than 2^8
+            // does some column need a (higher) reference?  first visible score, or a jump of more than 2^16
             if (soft_any(live && amax > RAISE_LOG2)) {
-                if (live) {
-#pragma unroll
-                    for (int ch = 0; ch < NCH; ++ch) {
-                        if (NCH > 1) {
-                            tmem_ld<CH>(s_addr + ch * CH, sv);
-                            tmem_wait_ld();
-                        }
-#pragma unroll
-                        for (int i = 0; i < CH; ++i) {
-                            float x = __uint_as_float(sv[i]) * c;
-                            if (NCH > 1 && masked && !((vis >> (ch * CH + i)) & 1)) x = -INFINITY;
-                            const int wm = __reduce_max_sync(0xffffffffu, ord_of(x));
-                            if (lane == 0) atomicMax(&cx.cmax[col0 + ch * CH + i], wm);
-                        }
-                    }
-                }
-                if (tid == 0) cx.flags[0] = 0;
-                soft_sync();
-                if (tid < NP) {
-                    const float mx = ord_to(cx.cmax[tid]);
-                    const float old = cx.mneg[tid];                    // -reference, or UNSET
-                    float al = 1.f;
-                    if (old == UNSET) {
-                        if (mx != -INFINITY) cx.mneg[tid] = -mx;
-                    } else if (mx > RAISE_LOG2 - old) {
-                        al = fast_exp2(-old - mx);
-                        cx.mneg[tid] = -mx;
-                        cx.flags[0] = 1;
-                    }
-                    cx.alpha[tid] = al;
-                    cx.cmax[tid] = INT_MIN;
-                }
-                soft_sync();
+                RaiseArgs ra;
+                ra.mneg = cx.mneg;
+                ra.abortp = cx.abortp;
+                ra.status = p.status;
+                ra.s_addr = s_addr;
+                ra.o_addr = cx.tmem + lane_base + TM_O + col0;
+                ra.pv_bar = cx.pv_done + 8 * ((g - 1) & 1);
+                ra.pv_parity = ((g - 1) >> 1) & 1;
+                ra.vis = vis;
+                ra.c = c;
+                ra.col0 = col0;
+                ra.live = live;
+                ra.rescale_o = t > 0;
+                ra.dead = dead;
+                const int rr = raise_references<NPH>(ra);
+                dead = (rr & 2) != 0;
 #pragma unroll
                 for (int i = 0; i < (REF_REGS ? NPH : 1); ++i) mr[i] = cx.mneg[col0 + i];
-                if (cx.flags[0]) {                                     // a reference moved: rescale sums and accumulator
+                if (rr & 1) {                                          // a reference moved: rescale the partial sums
 #pragma unroll
                     for (int i = 0; i < NPH; ++i) l[i] *= cx.alpha[col0 + i];
-                    if (t > 0) {
-                        wait_u(cx.pv_done + 8 * ((g - 1) & 1), ((g - 1) >> 1) & 1);   // no MMA may be writing O^T
-                        tc_fence_after();
-                        if (!dead) {
-#pragma unroll
-                            for (int ch = 0; ch < NCH; ++ch) {
-                                uint32_t ov[CH];
-                                tmem_ld<CH>(cx.tmem + lane_base + TM_O + col0 + ch * CH, ov);
-                                tmem_wait_ld();
-#pragma unroll
-                                for (int i = 0; i < CH; ++i) ov[i] = __float_as_uint(__uint_as_float(ov[i]) * cx.alpha[col0 + ch * CH + i]);
-                                tmem_st<CH>(cx.tmem + lane_base + TM_O + col0 + ch * CH, ov);
-                            }
-                            tmem_wait_st();
-                        }
-                    }
                 }
             }
             // the P^T buffer is still being read until the PV that used it last (two rounds ago, or
@@ -529,9 +604,12 @@ __device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& 
                     if (NCH > 1) {
                         tmem_ld<CH>(s_addr + ch * CH, sv);
                         tmem_wait_ld();
+                        if (masked) {
+                            const uint32_t vb = (uint32_t)(vis >> (ch * CH));
 #pragma unroll
-                        for (int i = 0; i < CH; ++i)
-                            if (masked && !((vis >> (ch * CH + i)) & 1)) sv[i] = 0xff800000u;
+                            for (int i = 0; i < CH; ++i)
+                                if (!((vb >> i) & 1)) sv[i] = 0xff800000u;
+                        }
                     }
 #pragma unroll
                     for (int j = 0; j < CH / 8; ++j) {
@@ -547,11 +625,11 @@ __device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& 
                     }
                 }
             }
-            if (!dead) {
-                tc_fence_before();
-                fence_async_smem();
-                mbar_arrive(cx.p_full + 8 * b);
-            }
+            // every thread orders its own TMEM reads and shared-memory writes, then one lane per warp signals
+            tc_fence_before();
+            fence_async_smem();
+            __syncwarp();
+            if (!dead && lane == 0) mbar_arrive(cx.p_full + 8 * b);
         }
     }
 #undef FDC_MNEG
@@ -587,10 +665,9 @@ __device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& 
         }
     }
     soft_sync();                     // column state and Q^T are free again
-    if (!dead) {
-        tc_fence_before();
-        mbar_arrive(cx.o_free);
-    }
+    tc_fence_before();
+    __syncwarp();
+    if (!dead && lane == 0) mbar_arrive(cx.o_free);
 }
 
 __global__ void __launch_bounds__(THREADS, 1)
@@ -648,11 +725,11 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, con
         }
         for (int i = 0; i < 2; ++i) {
             mbar_init(cx.s_full + 8 * i, 1);
-            mbar_init(cx.p_full + 8 * i, NSOFT * 32);
+            mbar_init(cx.p_full + 8 * i, NSOFT);
             mbar_init(cx.pv_done + 8 * i, 1);
         }
-        mbar_init(cx.q_ready, NSOFT * 32);
-        mbar_init(cx.o_free, NSOFT * 32);
+        mbar_init(cx.q_ready, NSOFT);
+        mbar_init(cx.o_free, NSOFT);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         fence_async_smem();
     }
