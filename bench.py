@@ -189,7 +189,7 @@ def run_fdc(args, rank: int, world: int):
         _build.build()
     if world > 1:
         dist.barrier()
-    from paper_2602_02864_b200 import fdc
+    from paper_2602_02864_b200 import fdc, replicas
     local = int(os.environ.get("LOCAL_RANK", 0))
     torch.cuda.set_device(local)
     device = torch.device("cuda", local)
@@ -198,7 +198,7 @@ def run_fdc(args, rank: int, world: int):
     def measure(name: str, K: int, W: int, with_e2e: bool, sample_clocks: bool):
         w = get_workload(name)
         total = W + K
-        sb = StepBench(w, total, device, seed_shift=rank)
+        sb = StepBench(w, total, device, seed_shift=replicas.replica_seed_shift(rank))
         ev = lambda: torch.cuda.Event(enable_timing=True)  # noqa: E731
         stream = torch.cuda.current_stream()
 
@@ -231,12 +231,8 @@ def run_fdc(args, rank: int, world: int):
         torch.cuda.synchronize()
         launches = fdc.fdc_launch_count() - l0
         clocks = sampler.stop() if sample_clocks else None
-        ms = e0.elapsed_time(e1)
-        if world > 1:
-            t = torch.tensor([ms], device=device, dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
-            dist.barrier()
+        ms = replicas.max_over_ranks(e0.elapsed_time(e1), device)      # the job's time: the slowest replica
+        replicas.barrier()
 
         # pass 2: per-launch duration of the dominant kernel (split-KV pass), CUDA events recorded by
         # the library itself on the launching stream around every such launch of the same K steps
@@ -287,11 +283,7 @@ def run_fdc(args, rank: int, world: int):
                 hout.copy_(sb.out, non_blocking=True)
             e1.record(stream)
             torch.cuda.synchronize()
-            ems = e0.elapsed_time(e1)
-            if world > 1:
-                t = torch.tensor([ems], device=device, dtype=torch.float64)
-                dist.all_reduce(t, op=dist.ReduceOp.MAX)
-                ems = float(t.item())
+            ems = replicas.max_over_ranks(e0.elapsed_time(e1), device)
             h2d = (dq.numel() + dk.numel() + dv.numel()) * w.esize
             d2h = sb.out.numel() * w.esize
             e2e = {"value": round(world * timed_bytes / (ems * 1e-3) / 1e9, 1), "unit": UNIT,

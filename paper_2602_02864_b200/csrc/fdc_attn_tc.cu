@@ -47,6 +47,7 @@ constexpr int STAGE = (D / 64) * PANEL;      // one K (or V) stage: 128 rows x h
 constexpr int MAXST = 4;                     // stages per ring at most
 constexpr float RAISE_LOG2 = 16.f;
 constexpr float UNSET = 1.0e30f;             // -reference of a column that has seen nothing yet
+constexpr int MBUF = 512;                    // bitmap words of a scene kept in shared memory (max_active * W)
 
 // ---------------------------------------------------------------- tcgen05 wrappers
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -159,6 +160,8 @@ struct Ctx {
     float *mneg, *alpha, *lred;      // [128] -reference per column, [128] rescale factors, [4][128] partial sums
     int *cmax, *flags;               // [128] column maxima (ordered ints), [2] flags of the raise path
     int *pre, *nact;                 // [batch + 1] tile prefix sums, [batch] active branches per scene
+    uint64_t* smask;                 // [MBUF] the current segment's scene bitmaps (when mstaged)
+    int mstaged;
     volatile int* abortp;
     int nk, nv, q_panel, p_buf, npb; // ring depths, bytes per 64-column panel of Q^T, bytes per P^T buffer, P^T buffers (1 or 2)
 };
@@ -167,6 +170,27 @@ struct Ctx {
 struct Round {
     int nt, tile0, tile1;
 };
+
+// Row bitmap (Eq. 1) of branch b of the segment's scene.  While the K/V stream saturates the
+// memory system a global read costs microseconds, so the softmax warps copy the scene's bitmaps
+// to shared memory at the start of a segment whenever they fit.
+__device__ __forceinline__ const uint64_t* mask_row(const AttnParams& p, const Ctx& cx, uint32_t seg, int s, int b)
+{
+    return cx.mstaged ? cx.smask + (seg & 1) * MBUF + (size_t)b * p.W : p.mask + ((size_t)s * p.max_active + b) * p.W;
+}
+// 16-byte asynchronous copy global -> shared (zero fill when !valid); completes with cp_async_wait_all.
+__device__ __forceinline__ void cp_async16(void* dst, const void* src, bool valid)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(smem_u32(dst)), "l"(src), "r"(valid ? 16 : 0) : "memory");
+}
+__device__ __forceinline__ void cp_async8(void* dst, const void* src)
+{
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(smem_u32(dst)), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all()
+{
+    asm volatile("cp.async.commit_group;\n\tcp.async.wait_group 0;" ::: "memory");
+}
 
 // One TMA producer warp: streams the K (or V) tiles of this CTA's units into its ring, two tiles
 // per stage (rows 0-63 and 64-127 of both 64-column panels).
@@ -286,6 +310,11 @@ __device__ __forceinline__ void pv_loop(const AttnParams& p, const Ctx& cx, long
         const int M = A * p.group;
         const int NP = M <= 16 ? 16 : (M <= 32 ? 32 : (M <= 64 ? 64 : 128));
         const uint32_t idesc_pv = instr_desc(D, NP, 1);
+        if (cx.mstaged) {                            // the softmax warps publish the scene's bitmaps with the queries
+            int okw = 1;
+            if (lane == 0) okw = mbar_wait(cx.q_ready, seg & 1, cx.abortp, p.status);
+            ok = __shfl_sync(0xffffffffu, okw, 0);
+        }
         int t = 0;
         for (int jb = sg.j0; jb < sg.j1 && ok; jb += 32) {
             const int jn = sg.j1 - jb < 32 ? sg.j1 - jb : 32;
@@ -303,7 +332,7 @@ __device__ __forceinline__ void pv_loop(const AttnParams& p, const Ctx& cx, long
                     if (tile * TILE + TILE <= p.P) continue;                 // all rows visible to everybody
                     uint64_t um = 0ull;
                     for (int b = lane; b < A; b += 32)
-                        um |= tile_rowmask(p.mask + ((size_t)sg.s * p.max_active + b) * p.W, p.W, p.P, tile);
+                        um |= tile_rowmask(mask_row(p, cx, seg, sg.s, b), p.W, p.P, tile);
                     const uint32_t ul = __reduce_or_sync(0xffffffffu, (uint32_t)um);
                     const uint32_t uh = __reduce_or_sync(0xffffffffu, (uint32_t)(um >> 32));
                     const uint64_t z = ~(((uint64_t)uh << 32) | ul);
@@ -468,8 +497,8 @@ __device__ __noinline__ int raise_references(const RaiseArgs a)
 
 // The softmax warps' work on one segment; NPH = query columns per thread (half of NP).
 template <int NPH>
-__device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& cx, const Segment& sg, uint32_t& g, bool& dead,
-                                                const int warp, const int lane)
+__device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& cx, const Segment& sg, const uint32_t seg, const long long hi,
+                                                int& prefetched, uint32_t& g, bool& dead, const int warp, const int lane)
 {
     constexpr int NP = 2 * NPH;
     constexpr int CH = NPH < 32 ? NPH : 32;       // columns handled at a time
@@ -489,15 +518,42 @@ __device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& 
     };
     // ---- Q^T (B operand of S^T = K Q^T): row n = query row, K-major, 128B swizzle, rows >= M zero
     {
-        const uint4* qg = reinterpret_cast<const uint4*>(p.q);
-        for (int idx = tid; idx < NP * (D / 8); idx += NSOFT * 32) {
-            const int n = idx / (D / 8), ch = idx - n * (D / 8);
-            uint4 v = make_uint4(0u, 0u, 0u, 0u);
-            if (n < M) {
-                const int b = n / G, hg = n - b * G;
-                v = qg[((((size_t)sg.s * p.max_active + b) * p.hq + (size_t)sg.g * G + hg) * D) / 8 + ch];
+        if (prefetched) {
+            // queries and bitmaps were copied asynchronously during the previous segment's last round
+            cp_async_wait_all();
+            prefetched = 0;
+        } else {
+            // all global reads first (one latency), then the stores
+            const uint4* qg = reinterpret_cast<const uint4*>(p.q);
+            uint4 qv[NP / 16];
+#pragma unroll
+            for (int i = 0; i < NP / 16; ++i) {
+                const int idx = tid + i * (NSOFT * 32);
+                const int n = idx / (D / 8), ch = idx - n * (D / 8);
+                qv[i] = make_uint4(0u, 0u, 0u, 0u);
+                if (n < M) {
+                    const int b = n / G, hg = n - b * G;
+                    qv[i] = qg[((((size_t)sg.s * p.max_active + b) * p.hq + (size_t)sg.g * G + hg) * D) / 8 + ch];
+                }
             }
-            *reinterpret_cast<uint4*>(cx.qs + (ch >> 3) * cx.q_panel + n * 128 + (((ch & 7) ^ (n & 7)) << 4)) = v;
+            uint64_t mv[MBUF / (NSOFT * 32)];
+            const int nw = cx.mstaged ? p.max_active * p.W : 0;
+#pragma unroll
+            for (int i = 0; i < MBUF / (NSOFT * 32); ++i) {
+                const int idx = tid + i * (NSOFT * 32);
+                mv[i] = idx < nw ? p.mask[(size_t)sg.s * p.max_active * p.W + idx] : 0ull;
+            }
+#pragma unroll
+            for (int i = 0; i < NP / 16; ++i) {
+                const int idx = tid + i * (NSOFT * 32);
+                const int n = idx / (D / 8), ch = idx - n * (D / 8);
+                *reinterpret_cast<uint4*>(cx.qs + (ch >> 3) * cx.q_panel + n * 128 + (((ch & 7) ^ (n & 7)) << 4)) = qv[i];
+            }
+#pragma unroll
+            for (int i = 0; i < MBUF / (NSOFT * 32); ++i) {
+                const int idx = tid + i * (NSOFT * 32);
+                if (idx < nw) cx.smask[(seg & 1) * MBUF + idx] = mv[i];
+            }
         }
         if (tid < NP) cx.mneg[tid] = UNSET;
         fence_async_smem();
@@ -531,8 +587,8 @@ __device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& 
             uint64_t vis = ~0ull;
             if (masked) {
                 uint64_t m0 = 0ull, m1 = 0ull;
-                if (lane < A) m0 = tile_rowmask(p.mask + ((size_t)sg.s * p.max_active + lane) * p.W, p.W, p.P, tile);
-                if (lane + 32 < A) m1 = tile_rowmask(p.mask + ((size_t)sg.s * p.max_active + lane + 32) * p.W, p.W, p.P, tile);
+                if (lane < A) m0 = tile_rowmask(mask_row(p, cx, seg, sg.s, lane), p.W, p.P, tile);
+                if (lane + 32 < A) m1 = tile_rowmask(mask_row(p, cx, seg, sg.s, lane + 32), p.W, p.P, tile);
                 // rows of this warp for branch `lane` / `lane + 32`
                 const uint32_t wlo = (q4 & 1) ? (uint32_t)(m0 >> 32) : (uint32_t)m0;
                 const uint32_t whi = (q4 & 1) ? (uint32_t)(m1 >> 32) : (uint32_t)m1;
@@ -550,6 +606,29 @@ __device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& 
             }
             wait_u(cx.s_full + 8 * b, (g >> 1) & 1);
             tc_fence_after();
+            if (jb + k + 2 >= ntile && sg.next_u < hi && !dead) {
+                // last round: every S^T = K Q^T of this segment has completed, so Q^T may be overwritten.
+                // The next segment's queries (and its scene's bitmaps, into the other buffer) are copied
+                // asynchronously; the latency hides behind this round, the drain and the partial write.
+                int s2 = sg.s;
+                const Segment nx = decode_segment(sg.next_u, hi, cx.pre, p.hkv, s2);
+                const int M2 = cx.nact[nx.s] * G;
+                const int NP2 = M2 <= 16 ? 16 : (M2 <= 32 ? 32 : (M2 <= 64 ? 64 : 128));
+                const uint4* qg = reinterpret_cast<const uint4*>(p.q);
+                for (int idx = tid; idx < NP2 * (D / 8); idx += NSOFT * 32) {
+                    const int n = idx / (D / 8), ch = idx - n * (D / 8);
+                    const bool valid = n < M2;
+                    const int bb = valid ? n / G : 0, hg = valid ? n - bb * G : 0;
+                    cp_async16(cx.qs + (ch >> 3) * cx.q_panel + n * 128 + (((ch & 7) ^ (n & 7)) << 4),
+                               qg + ((((size_t)nx.s * p.max_active + bb) * p.hq + (size_t)nx.g * G + hg) * D) / 8 + ch, valid);
+                }
+                if (cx.mstaged) {
+                    const uint64_t* src = p.mask + (size_t)nx.s * p.max_active * p.W;
+                    for (int idx = tid; idx < p.max_active * p.W; idx += NSOFT * 32)
+                        cp_async8(cx.smask + ((seg + 1) & 1) * MBUF + idx, src + idx);
+                }
+                prefetched = 1;
+            }
             const uint32_t s_addr = cx.tmem + lane_base + b * 128 + col0;
             uint32_t sv[CH];                       // raw scores of the current chunk (-inf where hidden)
             float amax = -INFINITY;                // max over this thread's columns of score * c - reference
@@ -670,6 +749,10 @@ __device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& 
     if (!dead && lane == 0) mbar_arrive(cx.o_free);
 }
 
+// NPMAX = query rows per (scene, KV head) the launch can meet, rounded up to 16/32/64/128: only
+// the softmax variants that can occur are compiled into a kernel, which keeps the register
+// allocation of the narrow ones free of the wide ones' pressure.
+template <int NPMAX>
 __global__ void __launch_bounds__(THREADS, 1)
 attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
                const int nk, const int nv, const int np_max, const int npb)
@@ -704,6 +787,8 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, con
     cx.flags = cx.cmax + 128;
     cx.pre = cx.flags + 4;
     cx.nact = cx.pre + p.batch + 1;
+    cx.smask = reinterpret_cast<uint64_t*>(((uintptr_t)(cx.nact + p.batch) + 7) & ~(uintptr_t)7);
+    cx.mstaged = p.max_active * p.W <= MBUF;
     __shared__ int abort_flag;
     cx.abortp = &abort_flag;
 
@@ -754,16 +839,23 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, con
         qk_loop(p, cx, lo, hi, lane);
     } else {
         int s = 0;
-        uint32_t g = 0;
+        uint32_t g = 0, seg = 0;
         long long u = lo;
         bool dead = false;                        // a bounded wait ran out somewhere in the CTA
+        int prefetched = 0;                       // the segment's queries and bitmaps are already on their way
         while (u < hi) {
             const Segment sg = decode_segment(u, hi, cx.pre, p.hkv, s);
             const int M = cx.nact[sg.s] * p.group;
-            if (M <= 16) softmax_segment<8>(p, cx, sg, g, dead, warp, lane);
-            else if (M <= 32) softmax_segment<16>(p, cx, sg, g, dead, warp, lane);
-            else if (M <= 64) softmax_segment<32>(p, cx, sg, g, dead, warp, lane);
-            else softmax_segment<64>(p, cx, sg, g, dead, warp, lane);
+            if (NPMAX == 16 || M <= 16) {
+                softmax_segment<8>(p, cx, sg, seg, hi, prefetched, g, dead, warp, lane);
+            } else if (NPMAX == 32 || M <= 32) {
+                if constexpr (NPMAX >= 32) softmax_segment<16>(p, cx, sg, seg, hi, prefetched, g, dead, warp, lane);
+            } else if (NPMAX == 64 || M <= 64) {
+                if constexpr (NPMAX >= 64) softmax_segment<32>(p, cx, sg, seg, hi, prefetched, g, dead, warp, lane);
+            } else {
+                if constexpr (NPMAX >= 128) softmax_segment<64>(p, cx, sg, seg, hi, prefetched, g, dead, warp, lane);
+            }
+            ++seg;
             u = sg.next_u;
         }
     }
@@ -789,24 +881,32 @@ int launch_attn_tc(const AttnParams& p, int head_dim, cudaStream_t st)
     const int p_buf = ((np_max + 63) / 64) * PANEL;
     const int npb = np_max > 64 ? 1 : 2;          // 128 query rows: one P^T buffer, so that four stages still fit
     const size_t fixed = 1024 + (size_t)npb * p_buf + (size_t)(D / 64) * np_max * 128 + 8 * (4 * MAXST + 8) + 16 +
-                         4 * (128 + 128 + 512 + 128 + 4) + sizeof(int) * (2 * p.batch + 1) + 64;
+                         4 * (128 + 128 + 512 + 128 + 4) + sizeof(int) * (2 * p.batch + 1) + 8 * (2 * MBUF + 2) + 64;
     int stages = (int)((227 * 1024 - 256 - fixed) / STAGE);
     if (stages > 2 * MAXST) stages = 2 * MAXST;
     if (stages < 4) return FDC_ERR_SHAPE;
     const int nk = stages / 2, nv = stages - nk;
     const size_t smem = fixed + (size_t)stages * STAGE;
-    static size_t attr_smem = 0;
-    if (smem > attr_smem) {
-        cudaError_t e = cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return set_cuda_error(e);
-        attr_smem = smem;
-    }
     alignas(64) CUtensorMap tk, tv;
     int rc = get_kv_tensor_map(p.k, p, D, TILE, &tk);
     if (rc) return rc;
     rc = get_kv_tensor_map(p.v, p, D, TILE, &tv);
     if (rc) return rc;
-    attn_tc_kernel<<<p.n_cta, THREADS, smem, st>>>(p, tk, tv, nk, nv, np_max, npb);
+    auto launch = [&](auto kernel, size_t& attr_smem) -> int {
+        if (smem > attr_smem) {
+            cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+            if (e != cudaSuccess) return set_cuda_error(e);
+            attr_smem = smem;
+        }
+        kernel<<<p.n_cta, THREADS, smem, st>>>(p, tk, tv, nk, nv, np_max, npb);
+        return FDC_OK;
+    };
+    static size_t attr16 = 0, attr32 = 0, attr64 = 0, attr128 = 0;
+    if (np_max == 16) rc = launch(attn_tc_kernel<16>, attr16);
+    else if (np_max == 32) rc = launch(attn_tc_kernel<32>, attr32);
+    else if (np_max == 64) rc = launch(attn_tc_kernel<64>, attr64);
+    else rc = launch(attn_tc_kernel<128>, attr128);
+    if (rc) return rc;
     note_launch();
     cudaError_t e = cudaGetLastError();
     return e == cudaSuccess ? FDC_OK : set_cuda_error(e);
