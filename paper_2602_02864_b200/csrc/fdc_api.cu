@@ -132,15 +132,16 @@ int fdc_plan_graph(const fdc_graph_desc* g, fdc_plan** out)
         p->sm_count = prop.multiProcessorCount;
         e = cudaMalloc((void**)&p->d, sizeof(PlanDev));
     }
-    if (e == cudaSuccess) e = cudaMalloc((void**)&p->d_status, 4 * sizeof(int32_t));
+    if (e == cudaSuccess) e = cudaMalloc((void**)&p->d_status, (4 + FDC_PAIR_COUNTERS) * sizeof(int32_t));
     if (e == cudaSuccess) e = cudaMemcpy(p->d, &p->h, sizeof(PlanDev), cudaMemcpyHostToDevice);
-    if (e == cudaSuccess) e = cudaMemset(p->d_status, 0, 4 * sizeof(int32_t));
+    if (e == cudaSuccess) e = cudaMemset(p->d_status, 0, (4 + FDC_PAIR_COUNTERS) * sizeof(int32_t));
     if (e != cudaSuccess) {
         int rc = set_cuda_error(e);
         fdc_plan_destroy(p);
         return rc;
     }
     p->d_ticket = p->d_status + 2;
+    p->d_pair_cnt = p->d_status + 4;
     *out = p;
     return FDC_OK;
 }
@@ -220,7 +221,11 @@ int fdc_status(const fdc_plan* p, int32_t* host_bits, int32_t clear, void* strea
     if (!p || !host_bits) return FDC_ERR_NULL;
     cudaStream_t st = (cudaStream_t)stream;
     FDC_CUDA(cudaMemcpyAsync(host_bits, p->d_status, sizeof(int32_t), cudaMemcpyDeviceToHost, st));
-    if (clear) FDC_CUDA(cudaMemsetAsync(p->d_status, 0, sizeof(int32_t), st));
+    if (clear) {
+        // a launch that gave up may have left arrival counters of the fused combine behind
+        FDC_CUDA(cudaMemsetAsync(p->d_status, 0, sizeof(int32_t), st));
+        FDC_CUDA(cudaMemsetAsync(p->d_pair_cnt, 0, FDC_PAIR_COUNTERS * sizeof(int32_t), st));
+    }
     FDC_CUDA(cudaStreamSynchronize(st));
     return *host_bits ? FDC_ERR_DEVICE : FDC_OK;
 }

@@ -160,13 +160,20 @@ int fdc_decode_attn(const fdc_plan* p, const fdc_kv_desc* kv, int32_t layer, con
         cudaEventRecord(e0, st);
     }
     rc = FDC_ERR_SHAPE;
-    if (kv->dtype == FDC_BF16 && (p->attn_kernel == 0 || p->attn_kernel == 3)) rc = launch_attn_tc(a, kv->head_dim, st);
+    a.pair_cnt = nullptr;
+    bool fused = false;                 // the split kernel merged the partials itself
+    if (kv->dtype == FDC_BF16 && (p->attn_kernel == 0 || p->attn_kernel == 3)) {
+        if ((long long)kv->batch * kv->hkv <= FDC_PAIR_COUNTERS) a.pair_cnt = p->d_pair_cnt;
+        rc = launch_attn_tc(a, kv->head_dim, st);
+        fused = rc == FDC_OK && a.pair_cnt != nullptr;
+        a.pair_cnt = nullptr;
+    }
     if (kv->dtype == FDC_BF16 && (p->attn_kernel == 2 || (rc == FDC_ERR_SHAPE && p->attn_kernel != 1)))
         rc = launch_attn_mma(a, kv->head_dim, st);
     if (rc == FDC_ERR_SHAPE) rc = launch_attn_ref(a, kv->dtype, kv->head_dim, st);
     if (rc) return rc;
     if (pr) cudaEventRecord(e1, st);
-    rc = launch_attn_combine(a, kv->dtype, kv->head_dim, st);
+    if (!fused) rc = launch_attn_combine(a, kv->dtype, kv->head_dim, st);
     if (pr) cudaEventRecord(e2, st);
     return rc;
 }

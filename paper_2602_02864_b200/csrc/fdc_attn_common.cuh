@@ -35,8 +35,10 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity)
     return ok != 0;
 }
 // Bounded wait: gives up after SPIN_LIMIT polls (or when another thread of the CTA gave up),
-// records FDC_DEV_TIMEOUT and returns false; the caller then skips all further work.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status)
+// records FDC_DEV_TIMEOUT and returns false; the caller then skips all further work.  The
+// polling loop is kept out of line: most waits are already satisfied when they are reached,
+// and the callers' loops stay small.
+static __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status)
 {
     for (uint32_t i = 0; i < SPIN_LIMIT; ++i) {
         if (mbar_try(bar, parity)) return true;
@@ -48,6 +50,11 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     *abort_flag = 1;
     atomicOr(status, 8 /* FDC_DEV_TIMEOUT */);
     return false;
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status)
+{
+    if (mbar_try(bar, parity)) return true;
+    return mbar_wait_slow(bar, parity, abort_flag, status);
 }
 __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int c0, int c1, int c2, int c3)
 {

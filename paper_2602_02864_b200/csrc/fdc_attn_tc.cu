@@ -47,6 +47,15 @@ constexpr int STAGE = (D / 64) * PANEL;      // one K (or V) stage: 128 rows x h
 constexpr int MAXST = 4;                     // stages per ring at most
 constexpr float RAISE_LOG2 = 16.f;
 constexpr float UNSET = 1.0e30f;             // -reference of a column that has seen nothing yet
+#ifndef FDC_W_MASKED
+#define FDC_W_MASKED 3
+#endif
+#ifndef FDC_W_PAIR
+#define FDC_W_PAIR 8
+#endif
+constexpr int W_MASKED = FDC_W_MASKED;       // cost of a tile beyond the prefix (bitmap selects, V clean-up) in prefix tiles
+constexpr int W_PAIR = FDC_W_PAIR;           // cost of finishing a (scene, KV head) pair (drain, partial write, next queries)
+constexpr int MIN_UNITS = 8;                 // tiles per CTA below which fewer CTAs are used (small problems)
 constexpr int MBUF = 512;                    // bitmap words of a scene kept in shared memory (max_active * W)
 
 // ---------------------------------------------------------------- tcgen05 wrappers
@@ -162,6 +171,10 @@ struct Ctx {
     int *pre, *nact;                 // [batch + 1] tile prefix sums, [batch] active branches per scene
     uint64_t* smask;                 // [MBUF] the current segment's scene bitmaps (when mstaged)
     int mstaged;
+    int n_cta;                       // CTAs that take part: at most the grid, at least MIN_UNITS tiles each
+    int* prev;                       // [batch + 1] prefix sums of the scenes' weighted lengths (per KV head), or nullptr
+    int npre;                        // tiles wholly inside the prefix
+    long long vtot;                  // total weighted length
     volatile int* abortp;
     int nk, nv, q_panel, p_buf, npb; // ring depths, bytes per 64-column panel of Q^T, bytes per P^T buffer, P^T buffers (1 or 2)
 };
@@ -190,6 +203,45 @@ __device__ __forceinline__ void cp_async8(void* dst, const void* src)
 __device__ __forceinline__ void cp_async_wait_all()
 {
     asm volatile("cp.async.commit_group;\n\tcp.async.wait_group 0;" ::: "memory");
+}
+
+// ---- weighted work split ---------------------------------------------------------------------
+// CTAs get equal shares of a WEIGHTED length, not of the tile count: a tile beyond the prefix
+// costs W_MASKED prefix tiles and the end of every pair costs W_PAIR.  Tile j of a pair starts at
+// weighted offset vt(j); a pair of nt tiles is vt(nt) + W_PAIR long.  A CTA owns the tiles whose
+// start falls into its share, so shares always cut the unit sequence into consecutive runs.
+__device__ __forceinline__ int vt_of(const Ctx& cx, int nt, int j)
+{
+    const int np = cx.npre < nt ? cx.npre : nt;
+    return j <= np ? j : np + (j - np) * W_MASKED;
+}
+// First unit whose weighted start is >= x.
+__device__ __forceinline__ long long unit_of_virt(const AttnParams& p, const Ctx& cx, long long x)
+{
+    if (x >= cx.vtot) return (long long)cx.pre[p.batch] * p.hkv;
+    int lo = 0, hi = p.batch;                      // largest s with prev[s] * hkv <= x
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if ((long long)cx.prev[mid] * p.hkv <= x) lo = mid;
+        else hi = mid;
+    }
+    int s = lo;
+    while (cx.prev[s + 1] == cx.prev[s]) ++s;     // scenes without tiles have no length
+    const int V = cx.prev[s + 1] - cx.prev[s], nt = cx.pre[s + 1] - cx.pre[s];
+    const long long y = x - (long long)cx.prev[s] * p.hkv;
+    const int g = (int)(y / V), r = (int)(y - (long long)g * V);
+    const int np = cx.npre < nt ? cx.npre : nt;
+    int j = r <= np ? r : np + (r - np + W_MASKED - 1) / W_MASKED;
+    if (j > nt) j = nt;
+    return (long long)cx.pre[s] * p.hkv + (long long)g * nt + j;
+}
+// CTA that owns tile j of pair (s, g).
+__device__ __forceinline__ int cta_of_tile(const AttnParams& p, const Ctx& cx, int s, int g, int j)
+{
+    const int nt = cx.pre[s + 1] - cx.pre[s];
+    if (!cx.prev) return unit_cta((long long)cx.pre[s] * p.hkv + (long long)g * nt + j, (long long)cx.pre[p.batch] * p.hkv, cx.n_cta);
+    const long long v = (long long)cx.prev[s] * p.hkv + (long long)g * (cx.prev[s + 1] - cx.prev[s]) + vt_of(cx, nt, j);
+    return (int)((v * cx.n_cta) / cx.vtot);
 }
 
 // One TMA producer warp: streams the K (or V) tiles of this CTA's units into its ring, two tiles
@@ -513,7 +565,8 @@ __device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& 
     const int M = A * p.group;
     const int G = p.group;
     auto wait_u = [&](uint32_t bar, uint32_t parity) {    // warp-uniform outcome
-        if (!dead && !mbar_wait(bar, parity, cx.abortp, p.status)) dead = true;
+        if (dead || __all_sync(0xffffffffu, mbar_try(bar, parity))) return;          // usually satisfied already
+        if (!mbar_wait_slow(bar, parity, cx.abortp, p.status)) dead = true;
         dead = __any_sync(0xffffffffu, dead);
     };
     // ---- Q^T (B operand of S^T = K Q^T): row n = query row, K-major, 128B swizzle, rows >= M zero
@@ -716,31 +769,154 @@ __device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& 
     const uint32_t last = g - 1;
     wait_u(cx.pv_done + 8 * (last & 1), (last >> 1) & 1);
     tc_fence_after();
+    // column sums over the warp's 32 rows by transpose-reduce: lane i ends up with column i's sum
 #pragma unroll
-    for (int i = 0; i < NPH; ++i) {
-        float x = l[i];
+    for (int ch = 0; ch < NCH; ++ch) {
+        float v[CH];
 #pragma unroll
-        for (int o = 16; o; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
-        if (lane == 0) cx.lred[q4 * 128 + col0 + i] = x;
+        for (int i = 0; i < CH; ++i) v[i] = l[ch * CH + i];
+#pragma unroll
+        for (int o = 16; o >= CH; o >>= 1)
+#pragma unroll
+            for (int i = 0; i < CH; ++i) v[i] += __shfl_xor_sync(0xffffffffu, v[i], o);
+#pragma unroll
+        for (int k = CH / 2; k >= 1; k >>= 1) {
+            const bool up = (lane & k) != 0;
+#pragma unroll
+            for (int i = 0; i < k; ++i) {
+                const float recv = __shfl_xor_sync(0xffffffffu, up ? v[i] : v[i + k], k);
+                v[i] = (up ? v[i + k] : v[i]) + recv;
+            }
+        }
+        if (lane < CH) cx.lred[q4 * 128 + col0 + ch * CH + lane] = v[0];
     }
     soft_sync();
-    const int slot = blockIdx.x + sg.s * p.hkv + sg.g;
-    if (!dead) {
-        if (tid < M) {
-            const float lt = (cx.lred[tid] + cx.lred[128 + tid]) + (cx.lred[256 + tid] + cx.lred[384 + tid]);
-            const float mn = cx.mneg[tid];
-            *reinterpret_cast<float2*>(p.ws_ml + ((size_t)slot * p.mmax + tid) * 2) = make_float2(mn == UNSET ? -INFINITY : -mn, lt);
+    const int pair = sg.s * p.hkv + sg.g;
+    const int slot = blockIdx.x + pair;
+    const bool whole = sg.j0 == 0 && sg.j1 == sg.nt;       // this CTA saw every tile of the pair
+    const uint32_t o_addr = cx.tmem + lane_base + TM_O + col0;
+    if (p.pair_cnt && whole) {
+        // no other partial exists: normalise and write the output directly
+        if (tid < NP) cx.alpha[tid] = 1.f / ((cx.lred[tid] + cx.lred[128 + tid]) + (cx.lred[256 + tid] + cx.lred[384 + tid]));
+        soft_sync();
+        if (!dead) {
+            __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(p.out);
+#pragma unroll
+            for (int ch = 0; ch < NCH; ++ch) {
+                uint32_t ov[CH];
+                tmem_ld<CH>(o_addr + ch * CH, ov);
+                tmem_wait_ld();
+                int b = (col0 + ch * CH) / G, hg = (col0 + ch * CH) - b * G;
+#pragma unroll
+                for (int i = 0; i < CH; ++i) {
+                    const int n = col0 + ch * CH + i;
+                    if (n < M)
+                        out[(((size_t)sg.s * p.max_active + b) * p.hq + (size_t)sg.g * G + hg) * D + krow] =
+                            __float2bfloat16_rn(__uint_as_float(ov[i]) * cx.alpha[n]);
+                    if (++hg == G) {
+                        hg = 0;
+                        ++b;
+                    }
+                }
+            }
         }
-        // O^T: lane = head_dim index, column = query row; partials are stored [query row][head_dim]
-        float* wo = p.ws_o + (size_t)slot * p.mmax * D + krow;
+    } else {
+        if (!dead) {
+            if (tid < M) {
+                const float lt = (cx.lred[tid] + cx.lred[128 + tid]) + (cx.lred[256 + tid] + cx.lred[384 + tid]);
+                const float mn = cx.mneg[tid];
+                *reinterpret_cast<float2*>(p.ws_ml + ((size_t)slot * p.mmax + tid) * 2) = make_float2(mn == UNSET ? -INFINITY : -mn, lt);
+            }
+            // O^T: lane = head_dim index, column = query row; partials are stored [query row][head_dim]
+            float* wo = p.ws_o + (size_t)slot * p.mmax * D + krow;
 #pragma unroll
-        for (int ch = 0; ch < NCH; ++ch) {
-            uint32_t ov[CH];
-            tmem_ld<CH>(cx.tmem + lane_base + TM_O + col0 + ch * CH, ov);
-            tmem_wait_ld();
+            for (int ch = 0; ch < NCH; ++ch) {
+                uint32_t ov[CH];
+                tmem_ld<CH>(o_addr + ch * CH, ov);
+                tmem_wait_ld();
 #pragma unroll
-            for (int i = 0; i < CH; ++i)
-                if (col0 + ch * CH + i < M) wo[(size_t)(col0 + ch * CH + i) * D] = __uint_as_float(ov[i]);
+                for (int i = 0; i < CH; ++i)
+                    if (col0 + ch * CH + i < M) wo[(size_t)(col0 + ch * CH + i) * D] = __uint_as_float(ov[i]);
+            }
+        }
+        if (p.pair_cnt) {
+            // the CTA that delivers the last partial of a pair merges them all (no second kernel)
+            __threadfence();
+            soft_sync();
+            if (tid == 0) {
+                const int c_first = cta_of_tile(p, cx, sg.s, sg.g, 0), c_last = cta_of_tile(p, cx, sg.s, sg.g, sg.nt - 1);
+                const int expected = c_last - c_first + 1;               // every CTA in between owns tiles of the pair
+                const int old = dead ? -1 : atomicAdd(&p.pair_cnt[pair], 1);
+                cx.flags[1] = old == expected - 1;
+                cx.flags[2] = c_first;
+                cx.flags[3] = c_last;
+                if (old == expected - 1) p.pair_cnt[pair] = 0;          // ready for the next call
+            }
+            soft_sync();
+            if (cx.flags[1]) {
+                __threadfence();
+                const int c_first = cx.flags[2], c_last = cx.flags[3];
+                // one thread per query row: m = max_c m_c, l = sum_c l_c 2^(m_c - m); the weight
+                // 2^(m_c - m) / l of every partial replaces m_c in the workspace.  Loads are issued
+                // four at a time: each costs a trip to L2 and nothing depends on the previous one.
+                if (tid < M) {
+                    float* ml = p.ws_ml + ((size_t)pair * p.mmax + tid) * 2;
+                    const size_t cs = (size_t)p.mmax * 2;                // stride between CTAs' entries
+                    float mx = -INFINITY;
+                    for (int c0 = c_first; c0 <= c_last; c0 += 4) {
+                        float v[4];
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) v[j] = c0 + j <= c_last ? __ldcg(ml + (size_t)(c0 + j) * cs) : -INFINITY;
+                        mx = fmaxf(fmaxf(mx, fmaxf(v[0], v[1])), fmaxf(v[2], v[3]));
+                    }
+                    float lt = 0.f;
+                    for (int c0 = c_first; c0 <= c_last; c0 += 4) {
+                        float2 v[4];
+#pragma unroll
+                        for (int j = 0; j < 4; ++j)
+                            v[j] = c0 + j <= c_last ? __ldcg(reinterpret_cast<const float2*>(ml + (size_t)(c0 + j) * cs)) : make_float2(-INFINITY, 0.f);
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) lt = fmaf(v[j].y, fast_exp2(v[j].x - mx), lt);   // a split that saw nothing: -inf -> 0
+                    }
+                    const float inv = 1.f / lt;
+                    for (int c = c_first; c <= c_last; ++c) {
+                        const float w = fast_exp2(__ldcg(ml + (size_t)c * cs) - mx) * inv;
+                        __stcg(ml + (size_t)c * cs, w);
+                    }
+                }
+                __threadfence();
+                soft_sync();
+                __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(p.out);
+                for (int idx = tid; idx < M * (D / 4); idx += NSOFT * 32) {
+                    const int m = idx / (D / 4), c4 = idx - m * (D / 4);
+                    const float* ml = p.ws_ml + ((size_t)pair * p.mmax + m) * 2;
+                    const float4* po = reinterpret_cast<const float4*>(p.ws_o + ((size_t)pair * p.mmax + m) * D) + c4;
+                    const size_t cs = (size_t)p.mmax * 2, os = (size_t)p.mmax * (D / 4);
+                    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+                    for (int c0 = c_first; c0 <= c_last; c0 += 4) {
+                        float w[4];
+                        float4 o[4];
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const bool on = c0 + j <= c_last;
+                            w[j] = on ? __ldcg(ml + (size_t)(c0 + j) * cs) : 0.f;
+                            o[j] = on ? __ldcg(po + (size_t)(c0 + j) * os) : make_float4(0.f, 0.f, 0.f, 0.f);
+                        }
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            acc.x = fmaf(o[j].x, w[j], acc.x);
+                            acc.y = fmaf(o[j].y, w[j], acc.y);
+                            acc.z = fmaf(o[j].z, w[j], acc.z);
+                            acc.w = fmaf(o[j].w, w[j], acc.w);
+                        }
+                    }
+                    const int b = m / G, hg = m - b * G;
+                    uint2 pk;
+                    pk.x = pack2(acc.x, acc.y);
+                    pk.y = pack2(acc.z, acc.w);
+                    *reinterpret_cast<uint2*>(out + (((size_t)sg.s * p.max_active + b) * p.hq + (size_t)sg.g * G + hg) * D + c4 * 4) = pk;
+                }
+            }
         }
     }
     soft_sync();                     // column state and Q^T are free again
@@ -787,7 +963,8 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, con
     cx.flags = cx.cmax + 128;
     cx.pre = cx.flags + 4;
     cx.nact = cx.pre + p.batch + 1;
-    cx.smask = reinterpret_cast<uint64_t*>(((uintptr_t)(cx.nact + p.batch) + 7) & ~(uintptr_t)7);
+    cx.prev = cx.nact + p.batch;
+    cx.smask = reinterpret_cast<uint64_t*>(((uintptr_t)(cx.prev + p.batch + 1) + 7) & ~(uintptr_t)7);
     cx.mstaged = p.max_active * p.W <= MBUF;
     __shared__ int abort_flag;
     cx.abortp = &abort_flag;
@@ -798,8 +975,46 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, con
     const long long total = scan_ntiles(p.ntiles, p.batch, cx.pre);
     const long long U = total * p.hkv;
     if (U == 0) return;
-    const long long lo = cta_first_unit(blockIdx.x, U, p.n_cta);
-    const long long hi = cta_first_unit(blockIdx.x + 1, U, p.n_cta);
+    // small problems use fewer CTAs (fewer partials to merge); every participating CTA owns units
+    {
+        // (only when this kernel also combines: a separate combine pass assumes the full grid)
+        const long long want = p.pair_cnt ? (U + MIN_UNITS - 1) / MIN_UNITS : p.n_cta;
+        cx.n_cta = (int)(want < p.n_cta ? want : p.n_cta);
+    }
+    if ((int)blockIdx.x >= cx.n_cta) return;
+    long long lo, hi;
+    if (p.pair_cnt) {
+        // weighted lengths of the scenes (one warp scans them)
+        cx.npre = p.P / TILE;
+        if (threadIdx.x < 32) {
+            int carry = 0;
+            for (int b0 = 0; b0 < p.batch; b0 += 32) {
+                const int i = b0 + threadIdx.x;
+                int x = 0;
+                if (i < p.batch) {
+                    const int nt = cx.pre[i + 1] - cx.pre[i];
+                    x = nt > 0 ? vt_of(cx, nt, nt) + W_PAIR : 0;
+                }
+                int inc = x;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const int y = __shfl_up_sync(0xffffffffu, inc, o);
+                    if ((int)threadIdx.x >= o) inc += y;
+                }
+                if (i < p.batch) cx.prev[i] = carry + inc - x;
+                carry += __shfl_sync(0xffffffffu, inc, 31);
+            }
+            if (threadIdx.x == 0) cx.prev[p.batch] = carry;
+        }
+        __syncthreads();
+        cx.vtot = (long long)cx.prev[p.batch] * p.hkv;
+        lo = unit_of_virt(p, cx, cta_first_unit(blockIdx.x, cx.vtot, cx.n_cta));
+        hi = unit_of_virt(p, cx, cta_first_unit(blockIdx.x + 1, cx.vtot, cx.n_cta));
+    } else {
+        cx.prev = nullptr;
+        lo = cta_first_unit(blockIdx.x, U, cx.n_cta);
+        hi = cta_first_unit(blockIdx.x + 1, U, cx.n_cta);
+    }
     if (lo >= hi) return;
     if (threadIdx.x == 0) {
         for (int i = 0; i < MAXST; ++i) {
@@ -881,7 +1096,7 @@ int launch_attn_tc(const AttnParams& p, int head_dim, cudaStream_t st)
     const int p_buf = ((np_max + 63) / 64) * PANEL;
     const int npb = np_max > 64 ? 1 : 2;          // 128 query rows: one P^T buffer, so that four stages still fit
     const size_t fixed = 1024 + (size_t)npb * p_buf + (size_t)(D / 64) * np_max * 128 + 8 * (4 * MAXST + 8) + 16 +
-                         4 * (128 + 128 + 512 + 128 + 4) + sizeof(int) * (2 * p.batch + 1) + 8 * (2 * MBUF + 2) + 64;
+                         4 * (128 + 128 + 512 + 128 + 4) + sizeof(int) * (3 * p.batch + 2) + 8 * (2 * MBUF + 2) + 64;
     int stages = (int)((227 * 1024 - 256 - fixed) / STAGE);
     if (stages > 2 * MAXST) stages = 2 * MAXST;
     if (stages < 4) return FDC_ERR_SHAPE;

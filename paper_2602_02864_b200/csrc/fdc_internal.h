@@ -6,6 +6,8 @@
 
 #include "fdc.h"
 
+#define FDC_PAIR_COUNTERS 65536
+
 namespace fdc {
 
 // Device-resident template tables (built on the host by fdc_plan_graph).
@@ -40,6 +42,7 @@ struct fdc_plan {
     fdc::PlanDev* d;                 // device copy
     int32_t*      d_status;          // sticky FDC_DEV_* bits
     int32_t*      d_ticket;          // [2] scratch of the frontier kernel's cross-block reduction
+    int32_t*      d_pair_cnt;        // [FDC_PAIR_COUNTERS] arrivals per (scene, KV head) of the fused combine (zero between calls)
     int           device;
     int           sm_count;
     int           attn_kernel;       // 0 auto
@@ -67,6 +70,7 @@ struct AttnParams {
     int32_t         batch, hkv, hq, group, max_active, mmax, W, P, rows, ntile_max, n_cta;
     float           scale_log2;      // softmax scale * log2(e)
     int32_t*        status;          // sticky FDC_DEV_* bits
+    int32_t*        pair_cnt;        // per (scene, KV head) arrival counters: the split kernel also combines (nullptr: it does not)
 };
 
 extern int64_t g_launches;
