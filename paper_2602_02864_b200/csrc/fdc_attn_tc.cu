@@ -441,6 +441,57 @@ __device__ __forceinline__ void pv_loop(const AttnParams& p, const Ctx& cx, long
     }
 }
 
+// Visibility (Eq. 1) of one KV row for the nph query columns starting at col0: bit i <=> column
+// col0 + i may see the row.  The warp's 32 rows are rows 32 * upper .. of tile `tile`; lane b first
+// extracts the rows' bits of branch b (and b + 32), then every lane collects its own row's bit of
+// the branches its columns belong to.  Kept out of line: only tiles beyond the prefix need it.
+__device__ __noinline__ uint64_t row_visibility(const uint64_t* mask0, int W, int P, int tile, int A, int G, int col0, int nph, int upper)
+{
+    const int lane = threadIdx.x & 31;
+    uint64_t m0 = 0ull, m1 = 0ull;
+    if (lane < A) m0 = tile_rowmask(mask0 + (size_t)lane * W, W, P, tile);
+    if (lane + 32 < A) m1 = tile_rowmask(mask0 + (size_t)(lane + 32) * W, W, P, tile);
+    const uint32_t wlo = upper ? (uint32_t)(m0 >> 32) : (uint32_t)m0;
+    const uint32_t whi = upper ? (uint32_t)(m1 >> 32) : (uint32_t)m1;
+    uint64_t vis = 0ull;
+    const int b_lo = col0 / G, b_hi = (col0 + nph - 1) / G;
+    for (int bq = b_lo; bq <= b_hi; ++bq) {
+        const uint32_t bits = __shfl_sync(0xffffffffu, bq < 32 ? wlo : whi, bq & 31);
+        if ((bits >> lane) & 1) {
+            const int c_lo = bq * G - col0 < 0 ? 0 : bq * G - col0;
+            const int c_hi = (bq + 1) * G - col0 > nph ? nph : (bq + 1) * G - col0;     // exclusive
+            const uint64_t span = c_hi - c_lo == 64 ? ~0ull : ((1ull << (c_hi - c_lo)) - 1ull);
+            vis |= span << c_lo;
+        }
+    }
+    return vis;
+}
+
+// Asynchronous copies of the next segment's queries into Q^T and of its scene's bitmaps into
+// the other bitmap buffer (softmax threads; completed with cp_async_wait_all in the prologue).
+// (All arguments by value: a reference to the caller's context would force it into local memory.)
+__device__ __noinline__ void prefetch_next_segment(const uint4* qg, const uint64_t* mask, int max_active, int W, int hq, int G, int hkv,
+                                                   const int* pre, const int* nact, unsigned char* qs, int q_panel,
+                                                   uint64_t* smask_dst, long long next_u, long long hi, int s_cur)
+{
+    const int tid = threadIdx.x;
+    int s2 = s_cur;
+    const Segment nx = decode_segment(next_u, hi, pre, hkv, s2);
+    const int M2 = nact[nx.s] * G;
+    const int NP2 = M2 <= 16 ? 16 : (M2 <= 32 ? 32 : (M2 <= 64 ? 64 : 128));
+    for (int idx = tid; idx < NP2 * (D / 8); idx += NSOFT * 32) {
+        const int n = idx / (D / 8), ch = idx - n * (D / 8);
+        const bool valid = n < M2;
+        const int bb = valid ? n / G : 0, hg = valid ? n - bb * G : 0;
+        cp_async16(qs + (ch >> 3) * q_panel + n * 128 + (((ch & 7) ^ (n & 7)) << 4),
+                   qg + ((((size_t)nx.s * max_active + bb) * hq + (size_t)nx.g * G + hg) * D) / 8 + ch, valid);
+    }
+    if (smask_dst) {
+        const uint64_t* src = mask + (size_t)nx.s * max_active * W;
+        for (int idx = tid; idx < max_active * W; idx += NSOFT * 32) cp_async8(smask_dst + idx, src + idx);
+    }
+}
+
 // The rare path of the softmax, kept out of line so that the per-round loop stays small: some
 // score exceeded its column's reference by more than 2^16 (or a column saw its first score).
 // Column maxima of the round are gathered (warp max, one shared-memory slot per warp), references
@@ -462,7 +513,7 @@ template <int NPH>
 __device__ __noinline__ int raise_references(const RaiseArgs a)
 {
     constexpr int NP = 2 * NPH;
-    constexpr int CH = NPH < 32 ? NPH : 32;
+    constexpr int CH = NPH < 16 ? NPH : 16;
     constexpr int NCH = NPH / CH;
     float* alpha = a.mneg + 128;
     int* wmax = reinterpret_cast<int*>(a.mneg + 256);      // [4][128]: maxima per row quadrant (shares the lred block)
@@ -553,7 +604,7 @@ __device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& 
                                                 int& prefetched, uint32_t& g, bool& dead, const int warp, const int lane)
 {
     constexpr int NP = 2 * NPH;
-    constexpr int CH = NPH < 32 ? NPH : 32;       // columns handled at a time
+    constexpr int CH = NPH < 16 ? NPH : 16;       // columns handled at a time
     constexpr int NCH = NPH / CH;
     const int tid = threadIdx.x;                  // 0..255
     const int q4 = warp & 3, half = warp >> 2;
@@ -637,49 +688,15 @@ __device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& 
             const bool live = ti < nt && !dead;                       // rows 64..127 of a one-tile round hold nothing
             const bool masked = live && tile * TILE + TILE > p.P;
             // Eq. 1 for this thread's KV row: bit i of vis <=> column col0 + i may see the row
-            uint64_t vis = ~0ull;
-            if (masked) {
-                uint64_t m0 = 0ull, m1 = 0ull;
-                if (lane < A) m0 = tile_rowmask(mask_row(p, cx, seg, sg.s, lane), p.W, p.P, tile);
-                if (lane + 32 < A) m1 = tile_rowmask(mask_row(p, cx, seg, sg.s, lane + 32), p.W, p.P, tile);
-                // rows of this warp for branch `lane` / `lane + 32`
-                const uint32_t wlo = (q4 & 1) ? (uint32_t)(m0 >> 32) : (uint32_t)m0;
-                const uint32_t whi = (q4 & 1) ? (uint32_t)(m1 >> 32) : (uint32_t)m1;
-                vis = 0ull;
-                const int b_lo = col0 / G, b_hi = (col0 + NPH - 1) / G;
-                for (int bq = b_lo; bq <= b_hi; ++bq) {
-                    const uint32_t bits = __shfl_sync(0xffffffffu, bq < 32 ? wlo : whi, bq & 31);
-                    if ((bits >> lane) & 1) {
-                        const int c_lo = bq * G - col0 < 0 ? 0 : bq * G - col0;
-                        const int c_hi = (bq + 1) * G - col0 > NPH ? NPH : (bq + 1) * G - col0;     // exclusive
-                        const uint64_t span = c_hi - c_lo == 64 ? ~0ull : ((1ull << (c_hi - c_lo)) - 1ull);
-                        vis |= span << c_lo;
-                    }
-                }
-            }
+            const uint64_t vis = masked ? row_visibility(mask_row(p, cx, seg, sg.s, 0), p.W, p.P, tile, A, G, col0, NPH, q4 & 1) : ~0ull;
             wait_u(cx.s_full + 8 * b, (g >> 1) & 1);
             tc_fence_after();
             if (jb + k + 2 >= ntile && sg.next_u < hi && !dead) {
                 // last round: every S^T = K Q^T of this segment has completed, so Q^T may be overwritten.
                 // The next segment's queries (and its scene's bitmaps, into the other buffer) are copied
                 // asynchronously; the latency hides behind this round, the drain and the partial write.
-                int s2 = sg.s;
-                const Segment nx = decode_segment(sg.next_u, hi, cx.pre, p.hkv, s2);
-                const int M2 = cx.nact[nx.s] * G;
-                const int NP2 = M2 <= 16 ? 16 : (M2 <= 32 ? 32 : (M2 <= 64 ? 64 : 128));
-                const uint4* qg = reinterpret_cast<const uint4*>(p.q);
-                for (int idx = tid; idx < NP2 * (D / 8); idx += NSOFT * 32) {
-                    const int n = idx / (D / 8), ch = idx - n * (D / 8);
-                    const bool valid = n < M2;
-                    const int bb = valid ? n / G : 0, hg = valid ? n - bb * G : 0;
-                    cp_async16(cx.qs + (ch >> 3) * cx.q_panel + n * 128 + (((ch & 7) ^ (n & 7)) << 4),
-                               qg + ((((size_t)nx.s * p.max_active + bb) * p.hq + (size_t)nx.g * G + hg) * D) / 8 + ch, valid);
-                }
-                if (cx.mstaged) {
-                    const uint64_t* src = p.mask + (size_t)nx.s * p.max_active * p.W;
-                    for (int idx = tid; idx < p.max_active * p.W; idx += NSOFT * 32)
-                        cp_async8(cx.smask + ((seg + 1) & 1) * MBUF + idx, src + idx);
-                }
+                prefetch_next_segment(reinterpret_cast<const uint4*>(p.q), p.mask, p.max_active, p.W, p.hq, G, p.hkv, cx.pre, cx.nact, cx.qs,
+                                      cx.q_panel, cx.mstaged ? cx.smask + ((seg + 1) & 1) * MBUF : nullptr, sg.next_u, hi, sg.s);
                 prefetched = 1;
             }
             const uint32_t s_addr = cx.tmem + lane_base + b * 128 + col0;
