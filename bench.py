@@ -28,6 +28,22 @@ import numpy as np
 ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
+# DRAM traffic of the split-KV kernel per algorithmic byte, from the ncu capture summarised in
+# profiles/attn_tc_kernel_cfg2.md (dram__bytes_read.sum + dram__bytes_write.sum over the launch's
+# algorithmic bytes; traffic grows in proportion to the visited tiles, so it scales to a full-size
+# launch).  Only valid for the kernel source it was measured on: keyed by a hash of that source.
+NCU_TRAFFIC = {"kernel_sha256_16": "d516ec6fb6ee4ebe", "dram_bytes_per_algorithmic_byte": 1.106}
+
+
+def kernel_source_hash() -> str:
+    import hashlib
+    path = os.path.join(ROOT, "paper_2602_02864_b200", "csrc", "fdc_attn_tc.cu")
+    try:
+        return hashlib.sha256(open(path, "rb").read()).hexdigest()[:16]
+    except OSError:
+        return ""
+
+
 METRIC = "masked_decode_attn_kv_bandwidth"
 UNIT = "GB/s"
 NOMINAL_HBM_GBS = 8000.0
@@ -251,9 +267,14 @@ def run_fdc(args, rank: int, world: int):
         if split_n:
             avg_bytes = timed_bytes / split_n
             achieved = avg_bytes / (split_ms / split_n * 1e-3) / 1e9
-            roof = {"kernel": prof["kernel"], "bound": "hbm", "achieved": round(achieved, 1), "peak": peak,
+            traffic = None
+            if w.dtype == "bf16" and w.head_dim == 128 and kernel_source_hash() == NCU_TRAFFIC["kernel_sha256_16"]:
+                traffic = int(avg_bytes * NCU_TRAFFIC["dram_bytes_per_algorithmic_byte"])
+            kname = ("attn_tc_kernel (tcgen05 split-KV pass, merges its partials itself)" if traffic is not None or
+                     (w.dtype == "bf16" and w.head_dim == 128) else "attn_ref_kernel (CUDA-core split-KV pass)")
+            roof = {"kernel": kname, "bound": "hbm", "achieved": round(achieved, 1), "peak": peak,
                     "unit": "GB/s", "frac": round(achieved / peak, 4), "peak_source": peak_src,
-                    "traffic": None, "launches": split_n, "avg_launch_us": round(split_ms / split_n * 1e3, 2),
+                    "traffic": traffic, "launches": split_n, "avg_launch_us": round(split_ms / split_n * 1e3, 2),
                     "algorithmic_bytes_per_launch": int(avg_bytes),
                     "combine_avg_launch_us": round(comb_ms / split_n * 1e3, 2),
                     "frac_of_nominal_8TBs": round(achieved / NOMINAL_HBM_GBS, 4)}

@@ -187,7 +187,10 @@ int fdc_attn_workspace_bytes(const fdc_plan* plan, const fdc_kv_desc* kv, size_t
  * softmax and accumulation are fp32; bf16 output is rounded to nearest even.  Each visited
  * KV tile is read once for all branches and all heads of its KV group; invisible K/V rows
  * may hold anything (NaN included).  d_workspace: DEVICE, 256-byte aligned,
- * >= fdc_attn_workspace_bytes; its contents are undefined afterwards. */
+ * >= fdc_attn_workspace_bytes; its contents are undefined afterwards.
+ * The tcgen05 kernel merges its split partials itself and keeps per-(scene, KV head) arrival
+ * counters in the plan: calls that use the same plan must be ordered on the GPU (one stream, or
+ * events); use one plan per concurrently decoding batch. */
 int fdc_decode_attn(const fdc_plan* plan, const fdc_kv_desc* kv, int32_t layer, const int32_t* d_n_active,
                     const uint64_t* d_mask, const int32_t* d_tiles, const int32_t* d_ntiles,
                     const void* d_q, void* d_out, float scale, void* d_workspace, size_t ws_bytes,
@@ -225,13 +228,14 @@ int fdc_decode_attn_static(const fdc_plan* plan, const fdc_kv_desc* kv, int32_t 
                            const uint64_t* d_mask, const int32_t* d_tiles, const int32_t* d_ntiles,
                            const void* d_q, void* d_out, float scale, void* stream);
 
-/* Reads (and with clear != 0 resets) the sticky device status word after synchronising
- * `stream`.  *host_bits receives the FDC_DEV_* bits; returns FDC_ERR_DEVICE if non-zero. */
+/* Reads (and with clear != 0 resets, together with the attention kernel's arrival counters,
+ * which a launch that gave up may have left behind) the sticky device status word after
+ * synchronising `stream`.  *host_bits receives the FDC_DEV_* bits; returns FDC_ERR_DEVICE if non-zero. */
 int fdc_status(const fdc_plan* plan, int32_t* host_bits, int32_t clear, void* stream);
 
 /* Selects the split-pass kernel: 0 = automatic (3 for bf16, 1 for fp32), 1 = CUDA-core kernel
- * (any dtype), 2 = TMA + mma.sync kernel (bf16), 3 = TMA + tcgen05/TMEM kernel (bf16).
- * Unsupported combinations use 1. */
+ * (any dtype), 2 = TMA + mma.sync kernel (bf16), 3 = TMA + tcgen05/TMEM kernel (bf16, head_dim
+ * 128; head_dim 64 takes 2).  Unsupported combinations use 1. */
 int fdc_set_attn_kernel(fdc_plan* plan, int32_t which);
 const char* fdc_kernel_name(int32_t which);
 
