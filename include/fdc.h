@@ -69,8 +69,11 @@ enum {
     FDC_DEV_FRONTIER_WIDE = 2,  /* fdc_frontier: more ready fields than max_active: clamped, */
                                 /* the others wait for a later pass                          */
     FDC_DEV_LEN_RANGE     = 4,  /* fdc_state_init: a length outside [n_fixed+1, C]: clamped  */
-    FDC_DEV_TIMEOUT       = 8   /* fdc_decode_attn: a bounded in-kernel wait ran out; the    */
+    FDC_DEV_TIMEOUT       = 8,  /* fdc_decode_attn: a bounded in-kernel wait ran out; the    */
                                 /* launch's output is invalid                                */
+    FDC_DEV_SCORE_RANGE   = 16  /* fdc_decode_attn: a score rose more than 2^100 above its   */
+                                /* softmax reference within two rounds (128 KV rows each)    */
+                                /* of a reference update: the output may have overflowed     */
 };
 
 typedef struct fdc_plan fdc_plan;

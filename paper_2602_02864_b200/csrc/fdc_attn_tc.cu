@@ -20,9 +20,9 @@
 //                columns.  Eq. 1 is applied by select from the branches' row bitmaps; prefix
 //                tiles skip it.
 // The softmax reference of a query column is raised lazily: it is set from the column maximum
-// of the first round (a column that sees no row yet borrows the round's highest maximum) and
-// raised again only when some score exceeds it by more than 2^16 (one barrier-wide OR per round
-// detects that).  Sum and accumulator use the same reference, so the
+// of the first round (a column that sees no row yet borrows the round's highest maximum).  A
+// score more than 2^16 above its reference leaves a note that all warps act on two rounds later
+// (no barrier in the common path); a rise of more than 2^100 within those two rounds is flagged.  Sum and accumulator use the same reference, so the
 // result is exact; the column sums are kept per thread and reduced at the end of a segment.
 #include <cudaTypedefs.h>
 
@@ -167,7 +167,8 @@ struct Ctx {
     uint32_t tmem;
     unsigned char *kring, *vring, *qs, *ps;
     float *mneg, *alpha, *lred;      // [128] -reference per column, [128] rescale factors, [4][128] partial sums
-    int *cmax, *flags;               // [128] column maxima (ordered ints), [2] flags of the raise path
+    int *cmax, *flags;               // [128] column maxima (ordered ints), [4] flags of the raise path and the merge
+    int* rflag;                      // [4] rflag[g & 3] == g: round g met a score far above its reference
     int *pre, *nact;                 // [batch + 1] tile prefix sums, [batch] active branches per scene
     uint64_t* smask;                 // [MBUF] the current segment's scene bitmaps (when mstaged)
     int mstaged;
@@ -699,6 +700,12 @@ __device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& 
                                       cx.q_panel, cx.mstaged ? cx.smask + ((seg + 1) & 1) * MBUF : nullptr, sg.next_u, hi, sg.s);
                 prefetched = 1;
             }
+            // The P^T buffer is still being read until the PV that used it last (two rounds ago, or the
+            // previous round when there is a single buffer) has completed.  Past this wait every softmax
+            // warp has also finished round g - 2, so what that round left in rflag is the same for all.
+            if (cx.npb == 2) wait_u(cx.pv_done + 8 * b, ((g >> 1) & 1) ^ 1);
+            else if (g > 0) wait_u(cx.pv_done + 8 * ((g - 1) & 1), ((g - 1) >> 1) & 1);
+            const bool do_raise = t == 0 || (g >= 2 && cx.rflag[(g - 2) & 3] == (int)(g - 2));
             const uint32_t s_addr = cx.tmem + lane_base + b * 128 + col0;
             uint32_t sv[CH];                       // raw scores of the current chunk (-inf where hidden)
             float amax = -INFINITY;                // max over this thread's columns of score * c - reference
@@ -717,8 +724,15 @@ __device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& 
                     for (int i = 0; i < CH; ++i) amax = fmaxf(amax, fmaf(__uint_as_float(sv[i]), c, FDC_MNEG(ch * CH + i)));
                 }
             }
-            // does some column need a (higher) reference?  first visible score, or a jump of more than 2^16
-            if (soft_any(live && amax > RAISE_LOG2)) {
+            // References are set in the first round of a segment.  Later a score more than 2^16 above its
+            // reference only leaves a note (no barrier in the common path): p stays far from overflow, and
+            // two rounds later, when all warps are known to see the note, the references are raised.
+            if (!do_raise) {
+                if (live && amax > RAISE_LOG2) {
+                    cx.rflag[g & 3] = (int)g;
+                    if (amax > 100.f) atomicOr(p.status, FDC_DEV_SCORE_RANGE);
+                }
+            } else {
                 RaiseArgs ra;
                 ra.mneg = cx.mneg;
                 ra.abortp = cx.abortp;
@@ -742,10 +756,6 @@ __device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& 
                     for (int i = 0; i < NPH; ++i) l[i] *= cx.alpha[col0 + i];
                 }
             }
-            // the P^T buffer is still being read until the PV that used it last (two rounds ago, or
-            // the previous round when there is a single buffer) has completed
-            if (cx.npb == 2) wait_u(cx.pv_done + 8 * b, ((g >> 1) & 1) ^ 1);
-            else if (g > 0) wait_u(cx.pv_done + 8 * ((g - 1) & 1), ((g - 1) >> 1) & 1);
             if (live) {
                 unsigned char* prow = cx.ps + (b & (cx.npb - 1)) * cx.p_buf + krow * 128;
 #pragma unroll
@@ -978,7 +988,8 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, con
     cx.lred = cx.alpha + 128;
     cx.cmax = reinterpret_cast<int*>(cx.lred + 512);
     cx.flags = cx.cmax + 128;
-    cx.pre = cx.flags + 4;
+    cx.rflag = cx.flags + 4;
+    cx.pre = cx.rflag + 4;
     cx.nact = cx.pre + p.batch + 1;
     cx.prev = cx.nact + p.batch;
     cx.smask = reinterpret_cast<uint64_t*>(((uintptr_t)(cx.prev + p.batch + 1) + 7) & ~(uintptr_t)7);
@@ -988,6 +999,7 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, con
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 0) abort_flag = 0;
+    if (threadIdx.x < 4) cx.rflag[threadIdx.x] = -1;
     for (int i = threadIdx.x; i < p.batch; i += THREADS) cx.nact[i] = p.n_active[i];
     const long long total = scan_ntiles(p.ntiles, p.batch, cx.pre);
     const long long U = total * p.hkv;
@@ -1113,7 +1125,7 @@ int launch_attn_tc(const AttnParams& p, int head_dim, cudaStream_t st)
     const int p_buf = ((np_max + 63) / 64) * PANEL;
     const int npb = np_max > 64 ? 1 : 2;          // 128 query rows: one P^T buffer, so that four stages still fit
     const size_t fixed = 1024 + (size_t)npb * p_buf + (size_t)(D / 64) * np_max * 128 + 8 * (4 * MAXST + 8) + 16 +
-                         4 * (128 + 128 + 512 + 128 + 4) + sizeof(int) * (3 * p.batch + 2) + 8 * (2 * MBUF + 2) + 64;
+                         4 * (128 + 128 + 512 + 128 + 8) + sizeof(int) * (3 * p.batch + 2) + 8 * (2 * MBUF + 2) + 64;
     int stages = (int)((227 * 1024 - 256 - fixed) / STAGE);
     if (stages > 2 * MAXST) stages = 2 * MAXST;
     if (stages < 4) return FDC_ERR_SHAPE;

@@ -169,3 +169,27 @@ def test_critical_path_host_call_matches_device_schedule():
             assert fin[v] == 1 + max(k for k, p in enumerate(passes) if any(x == v for x, _ in p))
         assert base.tolist() == sch.slot_base(w.slot_cap)
         fdc.fdc_plan_destroy(plan)
+
+
+def test_softmax_reference_is_raised_when_scores_jump(monkeypatch):
+    """Prefix keys that grow along the rows make later scores exceed the first rounds' maxima
+    by far more than 2^16: the kernel has to raise its softmax references and rescale sums and
+    accumulator in flight (deferred by two rounds), and must still match the checker."""
+    from paper_2602_02864_b200 import fdc
+    import harness
+    orig = wl.prefix_kv
+
+    def growing(w, layer, device="cpu", scenes=None):
+        k, v = orig(w, layer, device, scenes)
+        scale = torch.ones(w.prefix_len, device=k.device)
+        scale[300:] = 4.0
+        scale[700:] = 12.0
+        scale[1500:] = 0.25
+        k = (k.float() * scale[None, None, :, None]).to(k.dtype)
+        return k, v
+
+    monkeypatch.setattr(harness.wl, "prefix_kv", growing)
+    for branches in (4, 16):
+        w = wl.cfg4_sweep(2048, branches, 2)
+        r = run_and_compare(w, check_steps={0, 1, 2, 33, 63}, kernel=3)
+        assert r["checked"] > 0
