@@ -40,8 +40,9 @@ constexpr int RROWS = 2 * TILE;              // KV rows per round = M of S^T = K
 constexpr int NSOFT = 8;                     // softmax warps
 constexpr int W_KPROD = 8, W_QK = 9, W_VPROD = 10, W_PV = 11;
 constexpr int THREADS = 384;
-constexpr uint32_t TMEM_COLS = 512;          // S^T 0 [0,128) | S^T 1 [128,256) | O^T [256,384)
+constexpr uint32_t TMEM_COLS = 512;          // S^T 0 [0,128) | S^T 1 [128,256) | O^T [256,384) | sums [384,512)
 constexpr uint32_t TM_O = 256;
+constexpr uint32_t TM_L = 384;                // per-column sums of the softmax threads [384, 512)
 constexpr int PANEL = RROWS * 128;           // 128 rows x 128 bytes (64 bf16 columns)
 constexpr int STAGE = (D / 64) * PANEL;      // one K (or V) stage: 128 rows x head_dim
 constexpr int MAXST = 4;                     // stages per ring at most
@@ -493,52 +494,117 @@ __device__ __noinline__ void prefetch_next_segment(const uint4* qg, const uint64
     }
 }
 
-// The rare path of the softmax, kept out of line so that the per-round loop stays small: some
-// score exceeded its column's reference by more than 2^16 (or a column saw its first score).
-// Column maxima of the round are gathered (warp max, one shared-memory slot per warp), references
-// that are unset or too low are replaced, alpha[n] = 2^(old - new) is published, and the
-// accumulator O^T is rescaled when it already holds something.  Called by all softmax threads.
-// Returns bit 0: some reference moved (the caller rescales its partial sums by alpha),
-// bit 1: a bounded wait ran out.
+// Merge of the partials of one (scene, KV head) pair by the CTA that delivered the last one
+// (all softmax threads).  One thread per query row computes m = max_c m_c, l = sum_c l_c 2^(m_c - m)
+// and replaces m_c in the workspace by the weight 2^(m_c - m) / l; then every thread sums weighted
+// accumulator chunks.  Loads are issued four at a time: each costs a trip to L2 and none depends on
+// the previous one.  Out of line, arguments by value.
+__device__ __noinline__ void merge_pair(float* ws_ml, const float* ws_o, __nv_bfloat16* out, int pair, int mmax, int M, int G, int s, int g,
+                                        int max_active, int hq, int c_first, int c_last)
+{
+    const int tid = threadIdx.x;
+    __threadfence();
+    if (tid < M) {
+        float* ml = ws_ml + ((size_t)pair * mmax + tid) * 2;
+        const size_t cs = (size_t)mmax * 2;                // stride between CTAs' entries
+        float mx = -INFINITY;
+        for (int c0 = c_first; c0 <= c_last; c0 += 4) {
+            float v[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) v[j] = c0 + j <= c_last ? __ldcg(ml + (size_t)(c0 + j) * cs) : -INFINITY;
+            mx = fmaxf(fmaxf(mx, fmaxf(v[0], v[1])), fmaxf(v[2], v[3]));
+        }
+        float lt = 0.f;
+        for (int c0 = c_first; c0 <= c_last; c0 += 4) {
+            float2 v[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                v[j] = c0 + j <= c_last ? __ldcg(reinterpret_cast<const float2*>(ml + (size_t)(c0 + j) * cs)) : make_float2(-INFINITY, 0.f);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) lt = fmaf(v[j].y, fast_exp2(v[j].x - mx), lt);   // a split that saw nothing: -inf -> 0
+        }
+        const float inv = 1.f / lt;
+        for (int c = c_first; c <= c_last; ++c) {
+            const float w = fast_exp2(__ldcg(ml + (size_t)c * cs) - mx) * inv;
+            __stcg(ml + (size_t)c * cs, w);
+        }
+    }
+    __threadfence();
+    soft_sync();
+    for (int idx = tid; idx < M * (D / 4); idx += NSOFT * 32) {
+        const int m = idx / (D / 4), c4 = idx - m * (D / 4);
+        const float* ml = ws_ml + ((size_t)pair * mmax + m) * 2;
+        const float4* po = reinterpret_cast<const float4*>(ws_o + ((size_t)pair * mmax + m) * D) + c4;
+        const size_t cs = (size_t)mmax * 2, os = (size_t)mmax * (D / 4);
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int c0 = c_first; c0 <= c_last; c0 += 4) {
+            float w[4];
+            float4 o[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const bool on = c0 + j <= c_last;
+                w[j] = on ? __ldcg(ml + (size_t)(c0 + j) * cs) : 0.f;
+                o[j] = on ? __ldcg(po + (size_t)(c0 + j) * os) : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                acc.x = fmaf(o[j].x, w[j], acc.x);
+                acc.y = fmaf(o[j].y, w[j], acc.y);
+                acc.z = fmaf(o[j].z, w[j], acc.z);
+                acc.w = fmaf(o[j].w, w[j], acc.w);
+            }
+        }
+        const int b = m / G, hg = m - b * G;
+        uint2 pk;
+        pk.x = pack2(acc.x, acc.y);
+        pk.y = pack2(acc.z, acc.w);
+        *reinterpret_cast<uint2*>(out + (((size_t)s * max_active + b) * hq + (size_t)g * G + hg) * D + c4 * 4) = pk;
+    }
+}
+
+// The rare path of the softmax, kept out of line so that the per-round loop stays small: the
+// first round of a segment, or two rounds after some score exceeded its column's reference by
+// more than 2^16.  Column maxima of the round are gathered (shuffle transpose-reduce per warp,
+// one shared-memory slot per row quadrant), references that are unset or too low are replaced,
+// alpha[n] = 2^(old - new) is published, and the column sums (TMEM) and the accumulator O^T are
+// rescaled where a reference moved.  Called by all softmax threads.  Returns 1 when a bounded
+// wait ran out.  All arguments by value.
 struct RaiseArgs {
     float* mneg;                 // column state in shared memory: mneg[128], alpha[128], lred[512], cmax[128], flags[4]
     volatile int* abortp;
     int32_t* status;
-    uint32_t s_addr, o_addr;     // TMEM addresses of this thread's first score / accumulator column
+    uint32_t s_addr, o_addr, l_addr;   // TMEM addresses of this thread's first score / accumulator / sum column
     uint32_t pv_bar, pv_parity;  // completion of the previous round's O^T += V^T P^T
     uint64_t vis;                // Eq. 1 bits of this thread's columns
     float c;
-    int col0, live, rescale_o, dead;
+    int col0, nph, live, rescale_o, dead;
 };
-template <int NPH>
 __device__ __noinline__ int raise_references(const RaiseArgs a)
 {
-    constexpr int NP = 2 * NPH;
-    constexpr int CH = NPH < 16 ? NPH : 16;
-    constexpr int NCH = NPH / CH;
+    const int np = 2 * a.nph;
     float* alpha = a.mneg + 128;
     int* wmax = reinterpret_cast<int*>(a.mneg + 256);      // [4][128]: maxima per row quadrant (shares the lred block)
     int* flags = reinterpret_cast<int*>(a.mneg + 768) + 128;
     const int tid = threadIdx.x, lane = threadIdx.x & 31, q4 = (threadIdx.x >> 5) & 3;
     bool dead = a.dead != 0;
-#pragma unroll
-    for (int ch = 0; ch < NCH; ++ch) {
-        float mine = -INFINITY;                              // lane i ends up with the maximum of column ch * CH + i
+    for (int ch = 0; ch < a.nph / 8; ++ch) {
+        float mine = -INFINITY;                              // lane i < 8 ends up with the maximum of column ch * 8 + i
         if (a.live) {
-            uint32_t sv[CH];
-            tmem_ld<CH>(a.s_addr + ch * CH, sv);
+            uint32_t sv[8];
+            tmem_ld<8>(a.s_addr + ch * 8, sv);
             tmem_wait_ld();
-            float v[CH];
+            float v[8];
+            const uint32_t vb = (uint32_t)(a.vis >> (ch * 8));
 #pragma unroll
-            for (int i = 0; i < CH; ++i) v[i] = ((a.vis >> (ch * CH + i)) & 1) ? __uint_as_float(sv[i]) * a.c : -INFINITY;
-            // lanes whose index differs in bits >= CH hold rows of the same columns: plain max
+            for (int i = 0; i < 8; ++i) v[i] = ((vb >> i) & 1) ? __uint_as_float(sv[i]) * a.c : -INFINITY;
+            // lanes whose index differs in bits >= 8 hold rows of the same columns: plain max
 #pragma unroll
-            for (int o = 16; o >= CH; o >>= 1)
+            for (int o = 16; o >= 8; o >>= 1)
 #pragma unroll
-                for (int i = 0; i < CH; ++i) v[i] = fmaxf(v[i], __shfl_xor_sync(0xffffffffu, v[i], o));
+                for (int i = 0; i < 8; ++i) v[i] = fmaxf(v[i], __shfl_xor_sync(0xffffffffu, v[i], o));
             // transpose-reduce: at distance k a lane keeps the half of the columns that matches its bit k
 #pragma unroll
-            for (int k = CH / 2; k >= 1; k >>= 1) {
+            for (int k = 4; k >= 1; k >>= 1) {
                 const bool up = (lane & k) != 0;
 #pragma unroll
                 for (int i = 0; i < k; ++i) {
@@ -548,18 +614,18 @@ __device__ __noinline__ int raise_references(const RaiseArgs a)
             }
             mine = v[0];
         }
-        if (lane < CH) wmax[q4 * 128 + a.col0 + ch * CH + lane] = ord_of(mine);
+        if (lane < 8) wmax[q4 * 128 + a.col0 + ch * 8 + lane] = ord_of(mine);
     }
     if (tid == 0) flags[0] = 0;
     soft_sync();
-    if (tid < ((NP + 31) & ~31)) {                         // whole warps (the shuffles below need all lanes)
+    if (tid < ((np + 31) & ~31)) {                         // whole warps (the shuffles below need all lanes)
         // highest column maximum of the round (every warp of these threads computes it for itself)
         int gm = INT_MIN;
-        for (int n = lane; n < NP; n += 32)
+        for (int n = lane; n < np; n += 32)
             gm = max(gm, max(max(wmax[n], wmax[128 + n]), max(wmax[256 + n], wmax[384 + n])));
 #pragma unroll
         for (int o = 16; o; o >>= 1) gm = max(gm, __shfl_xor_sync(0xffffffffu, gm, o));
-        if (tid < NP) {
+        if (tid < np) {
             const int m01 = max(wmax[tid], wmax[128 + tid]), m23 = max(wmax[256 + tid], wmax[384 + tid]);
             const float mx = ord_to(max(m01, m23));
             const float old = a.mneg[tid];                     // -reference, or UNSET
@@ -578,44 +644,54 @@ __device__ __noinline__ int raise_references(const RaiseArgs a)
         }
     }
     soft_sync();
-    const int moved = flags[0];
-    if (moved && a.rescale_o) {
-        if (!dead && !mbar_wait(a.pv_bar, a.pv_parity, a.abortp, a.status)) dead = true;   // no MMA may be writing O^T
-        dead = __any_sync(0xffffffffu, dead);
-        tc_fence_after();
-        if (!dead) {
+    if (flags[0]) {                                        // a reference moved: rescale sums and accumulator
+        for (int ch = 0; ch < a.nph / 8; ++ch) {
+            uint32_t lv[8];
+            tmem_ld<8>(a.l_addr + ch * 8, lv);
+            tmem_wait_ld();
 #pragma unroll
-            for (int ch = 0; ch < NCH; ++ch) {
-                uint32_t ov[CH];
-                tmem_ld<CH>(a.o_addr + ch * CH, ov);
-                tmem_wait_ld();
-#pragma unroll
-                for (int i = 0; i < CH; ++i) ov[i] = __float_as_uint(__uint_as_float(ov[i]) * alpha[a.col0 + ch * CH + i]);
-                tmem_st<CH>(a.o_addr + ch * CH, ov);
-            }
-            tmem_wait_st();
+            for (int i = 0; i < 8; ++i) lv[i] = __float_as_uint(__uint_as_float(lv[i]) * alpha[a.col0 + ch * 8 + i]);
+            tmem_st<8>(a.l_addr + ch * 8, lv);
         }
+        if (a.rescale_o) {
+            if (!dead && !mbar_wait(a.pv_bar, a.pv_parity, a.abortp, a.status)) dead = true;   // no MMA may be writing O^T
+            dead = __any_sync(0xffffffffu, dead);
+            tc_fence_after();
+            if (!dead) {
+                for (int ch = 0; ch < a.nph / 8; ++ch) {
+                    uint32_t ov[8];
+                    tmem_ld<8>(a.o_addr + ch * 8, ov);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) ov[i] = __float_as_uint(__uint_as_float(ov[i]) * alpha[a.col0 + ch * 8 + i]);
+                    tmem_st<8>(a.o_addr + ch * 8, ov);
+                }
+            }
+        }
+        tmem_wait_st();
     }
-    return moved | (dead ? 2 : 0);
+    return dead ? 1 : 0;
 }
 
-// The softmax warps' work on one segment; NPH = query columns per thread (half of NP).
-template <int NPH>
-__device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& cx, const Segment& sg, const uint32_t seg, const long long hi,
-                                                int& prefetched, uint32_t& g, bool& dead, const int warp, const int lane)
+// The softmax warps' work on one segment; nph = query columns per thread (half of NP: 8, 16, 32
+// or 64).  Columns are handled eight at a time in real loops, with the per-column sums kept in
+// TMEM (the free columns [384, 512)) and the references read from shared memory, so that the
+// same small loop serves every width.
+__device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& cx, const Segment& sg, const int nph, const uint32_t seg,
+                                                const long long hi, int& prefetched, uint32_t& g, bool& dead, const int warp, const int lane)
 {
-    constexpr int NP = 2 * NPH;
-    constexpr int CH = NPH < 16 ? NPH : 16;       // columns handled at a time
-    constexpr int NCH = NPH / CH;
+    const int np = 2 * nph, nch = nph >> 3;
     const int tid = threadIdx.x;                  // 0..255
     const int q4 = warp & 3, half = warp >> 2;
     const int krow = q4 * 32 + lane;              // KV row of the round = TMEM lane of S^T; head_dim index for O^T
     const uint32_t lane_base = (uint32_t)(q4 * 32) << 16;
-    const int col0 = half * NPH;
+    const int col0 = half * nph;
     const float c = p.scale_log2;
     const int A = cx.nact[sg.s];
     const int M = A * p.group;
     const int G = p.group;
+    const uint32_t o_addr = cx.tmem + lane_base + TM_O + col0;
+    const uint32_t l_addr = cx.tmem + lane_base + TM_L + col0;
     auto wait_u = [&](uint32_t bar, uint32_t parity) {    // warp-uniform outcome
         if (dead || __all_sync(0xffffffffu, mbar_try(bar, parity))) return;          // usually satisfied already
         if (!mbar_wait_slow(bar, parity, cx.abortp, p.status)) dead = true;
@@ -630,9 +706,9 @@ __device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& 
         } else {
             // all global reads first (one latency), then the stores
             const uint4* qg = reinterpret_cast<const uint4*>(p.q);
-            uint4 qv[NP / 16];
+            uint4 qv[8];
 #pragma unroll
-            for (int i = 0; i < NP / 16; ++i) {
+            for (int i = 0; i < 8; ++i) {
                 const int idx = tid + i * (NSOFT * 32);
                 const int n = idx / (D / 8), ch = idx - n * (D / 8);
                 qv[i] = make_uint4(0u, 0u, 0u, 0u);
@@ -649,10 +725,10 @@ __device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& 
                 mv[i] = idx < nw ? p.mask[(size_t)sg.s * p.max_active * p.W + idx] : 0ull;
             }
 #pragma unroll
-            for (int i = 0; i < NP / 16; ++i) {
+            for (int i = 0; i < 8; ++i) {
                 const int idx = tid + i * (NSOFT * 32);
                 const int n = idx / (D / 8), ch = idx - n * (D / 8);
-                *reinterpret_cast<uint4*>(cx.qs + (ch >> 3) * cx.q_panel + n * 128 + (((ch & 7) ^ (n & 7)) << 4)) = qv[i];
+                if (n < np) *reinterpret_cast<uint4*>(cx.qs + (ch >> 3) * cx.q_panel + n * 128 + (((ch & 7) ^ (n & 7)) << 4)) = qv[i];
             }
 #pragma unroll
             for (int i = 0; i < MBUF / (NSOFT * 32); ++i) {
@@ -660,21 +736,19 @@ __device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& 
                 if (idx < nw) cx.smask[(seg & 1) * MBUF + idx] = mv[i];
             }
         }
-        if (tid < NP) cx.mneg[tid] = UNSET;
+        if (tid < np) cx.mneg[tid] = UNSET;
+        {
+            uint32_t z[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) z[i] = 0u;
+            for (int ch = 0; ch < nch; ++ch) tmem_st<8>(l_addr + ch * 8, z);      // column sums start at 0
+            tmem_wait_st();
+        }
         fence_async_smem();
         __syncwarp();
         if (!dead && lane == 0) mbar_arrive(cx.q_ready);
         soft_sync();
     }
-    float l[NPH];
-#pragma unroll
-    for (int i = 0; i < NPH; ++i) l[i] = 0.f;
-    // -reference of this thread's columns: in registers when they fit, else read from shared memory
-    constexpr bool REF_REGS = NPH <= 32;
-    float mr[REF_REGS ? NPH : 1];
-#pragma unroll
-    for (int i = 0; i < (REF_REGS ? NPH : 1); ++i) mr[i] = UNSET;
-#define FDC_MNEG(i) (REF_REGS ? mr[REF_REGS ? (i) : 0] : cx.mneg[col0 + (i)])
 
     const int ntile = sg.j1 - sg.j0;
     int t = 0;                                    // round within the segment
@@ -689,7 +763,7 @@ __device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& 
             const bool live = ti < nt && !dead;                       // rows 64..127 of a one-tile round hold nothing
             const bool masked = live && tile * TILE + TILE > p.P;
             // Eq. 1 for this thread's KV row: bit i of vis <=> column col0 + i may see the row
-            const uint64_t vis = masked ? row_visibility(mask_row(p, cx, seg, sg.s, 0), p.W, p.P, tile, A, G, col0, NPH, q4 & 1) : ~0ull;
+            const uint64_t vis = masked ? row_visibility(mask_row(p, cx, seg, sg.s, 0), p.W, p.P, tile, A, G, col0, nph, q4 & 1) : ~0ull;
             wait_u(cx.s_full + 8 * b, (g >> 1) & 1);
             tc_fence_after();
             if (jb + k + 2 >= ntile && sg.next_u < hi && !dead) {
@@ -705,83 +779,63 @@ __device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& 
             // warp has also finished round g - 2, so what that round left in rflag is the same for all.
             if (cx.npb == 2) wait_u(cx.pv_done + 8 * b, ((g >> 1) & 1) ^ 1);
             else if (g > 0) wait_u(cx.pv_done + 8 * ((g - 1) & 1), ((g - 1) >> 1) & 1);
-            const bool do_raise = t == 0 || (g >= 2 && cx.rflag[(g - 2) & 3] == (int)(g - 2));
             const uint32_t s_addr = cx.tmem + lane_base + b * 128 + col0;
-            uint32_t sv[CH];                       // raw scores of the current chunk (-inf where hidden)
-            float amax = -INFINITY;                // max over this thread's columns of score * c - reference
-            if (live) {
-#pragma unroll
-                for (int ch = 0; ch < NCH; ++ch) {
-                    tmem_ld<CH>(s_addr + ch * CH, sv);
-                    tmem_wait_ld();
-                    if (masked) {                                      // uniform branch: prefix rounds skip the selects
-                        const uint32_t vb = (uint32_t)(vis >> (ch * CH));
-#pragma unroll
-                        for (int i = 0; i < CH; ++i)
-                            if (!((vb >> i) & 1)) sv[i] = 0xff800000u;
-                    }
-#pragma unroll
-                    for (int i = 0; i < CH; ++i) amax = fmaxf(amax, fmaf(__uint_as_float(sv[i]), c, FDC_MNEG(ch * CH + i)));
-                }
-            }
             // References are set in the first round of a segment.  Later a score more than 2^16 above its
             // reference only leaves a note (no barrier in the common path): p stays far from overflow, and
             // two rounds later, when all warps are known to see the note, the references are raised.
-            if (!do_raise) {
-                if (live && amax > RAISE_LOG2) {
-                    cx.rflag[g & 3] = (int)g;
-                    if (amax > 100.f) atomicOr(p.status, FDC_DEV_SCORE_RANGE);
-                }
-            } else {
+            if (t == 0 || (g >= 2 && cx.rflag[(g - 2) & 3] == (int)(g - 2))) {
                 RaiseArgs ra;
                 ra.mneg = cx.mneg;
                 ra.abortp = cx.abortp;
                 ra.status = p.status;
                 ra.s_addr = s_addr;
-                ra.o_addr = cx.tmem + lane_base + TM_O + col0;
+                ra.o_addr = o_addr;
+                ra.l_addr = l_addr;
                 ra.pv_bar = cx.pv_done + 8 * ((g - 1) & 1);
                 ra.pv_parity = ((g - 1) >> 1) & 1;
                 ra.vis = vis;
                 ra.c = c;
                 ra.col0 = col0;
+                ra.nph = nph;
                 ra.live = live;
                 ra.rescale_o = t > 0;
                 ra.dead = dead;
-                const int rr = raise_references<NPH>(ra);
-                dead = (rr & 2) != 0;
-#pragma unroll
-                for (int i = 0; i < (REF_REGS ? NPH : 1); ++i) mr[i] = cx.mneg[col0 + i];
-                if (rr & 1) {                                          // a reference moved: rescale the partial sums
-#pragma unroll
-                    for (int i = 0; i < NPH; ++i) l[i] *= cx.alpha[col0 + i];
-                }
+                dead = raise_references(ra) != 0;
             }
             if (live) {
                 unsigned char* prow = cx.ps + (b & (cx.npb - 1)) * cx.p_buf + krow * 128;
+                float emax = 0.f;
+#pragma unroll 1
+                for (int ch = 0; ch < nch; ++ch) {
+                    uint32_t sv[8], lv[8];
+                    tmem_ld<8>(s_addr + ch * 8, sv);
+                    tmem_ld<8>(l_addr + ch * 8, lv);
+                    const float4 m0 = *reinterpret_cast<const float4*>(cx.mneg + col0 + ch * 8);
+                    const float4 m1 = *reinterpret_cast<const float4*>(cx.mneg + col0 + ch * 8 + 4);
+                    const float mn[8] = {m0.x, m0.y, m0.z, m0.w, m1.x, m1.y, m1.z, m1.w};
+                    tmem_wait_ld();
+                    if (masked) {                                      // uniform branch: prefix rounds skip the selects
+                        const uint32_t vb = (uint32_t)(vis >> (ch * 8));
 #pragma unroll
-                for (int ch = 0; ch < NCH; ++ch) {
-                    if (NCH > 1) {
-                        tmem_ld<CH>(s_addr + ch * CH, sv);
-                        tmem_wait_ld();
-                        if (masked) {
-                            const uint32_t vb = (uint32_t)(vis >> (ch * CH));
-#pragma unroll
-                            for (int i = 0; i < CH; ++i)
-                                if (!((vb >> i) & 1)) sv[i] = 0xff800000u;
-                        }
+                        for (int i = 0; i < 8; ++i)
+                            if (!((vb >> i) & 1)) sv[i] = 0xff800000u;
                     }
+                    float e[8];
 #pragma unroll
-                    for (int j = 0; j < CH / 8; ++j) {
-                        float e[8];
-#pragma unroll
-                        for (int i = 0; i < 8; ++i) {
-                            e[i] = fast_exp2(fmaf(__uint_as_float(sv[j * 8 + i]), c, FDC_MNEG(ch * CH + j * 8 + i)));
-                            l[ch * CH + j * 8 + i] += e[i];
-                        }
-                        const int cidx = (col0 + ch * CH) / 8 + j;     // 16-byte chunk of the P^T row
-                        *reinterpret_cast<uint4*>(prow + (cidx >> 3) * PANEL + (((cidx & 7) ^ (krow & 7)) << 4)) =
-                            make_uint4(pack2(e[0], e[1]), pack2(e[2], e[3]), pack2(e[4], e[5]), pack2(e[6], e[7]));
+                    for (int i = 0; i < 8; ++i) {
+                        e[i] = fast_exp2(fmaf(__uint_as_float(sv[i]), c, mn[i]));
+                        emax = fmaxf(emax, e[i]);
+                        lv[i] = __float_as_uint(__uint_as_float(lv[i]) + e[i]);
                     }
+                    tmem_st<8>(l_addr + ch * 8, lv);
+                    const int cidx = (col0 >> 3) + ch;                 // 16-byte chunk of the P^T row
+                    *reinterpret_cast<uint4*>(prow + (cidx >> 3) * PANEL + (((cidx & 7) ^ (krow & 7)) << 4)) =
+                        make_uint4(pack2(e[0], e[1]), pack2(e[2], e[3]), pack2(e[4], e[5]), pack2(e[6], e[7]));
+                }
+                tmem_wait_st();
+                if (emax > 65536.f) {                                  // 2^16 above the reference: note it for round g + 2
+                    cx.rflag[g & 3] = (int)g;
+                    if (!(emax < 1.0e30f)) atomicOr(p.status, FDC_DEV_SCORE_RANGE);     // beyond 2^100 (or inf / nan)
                 }
             }
             // every thread orders its own TMEM reads and shared-memory writes, then one lane per warp signals
@@ -791,23 +845,25 @@ __device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& 
             if (!dead && lane == 0) mbar_arrive(cx.p_full + 8 * b);
         }
     }
-#undef FDC_MNEG
     // ---- end of segment: the accumulator is final once the last PV has completed
     const uint32_t last = g - 1;
     wait_u(cx.pv_done + 8 * (last & 1), (last >> 1) & 1);
     tc_fence_after();
-    // column sums over the warp's 32 rows by transpose-reduce: lane i ends up with column i's sum
+    // column sums over the warp's 32 rows by transpose-reduce: lane i < 8 ends up with column i's sum
+#pragma unroll 1
+    for (int ch = 0; ch < nch; ++ch) {
+        uint32_t lv[8];
+        tmem_ld<8>(l_addr + ch * 8, lv);
+        tmem_wait_ld();
+        float v[8];
 #pragma unroll
-    for (int ch = 0; ch < NCH; ++ch) {
-        float v[CH];
+        for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(lv[i]);
 #pragma unroll
-        for (int i = 0; i < CH; ++i) v[i] = l[ch * CH + i];
+        for (int o = 16; o >= 8; o >>= 1)
 #pragma unroll
-        for (int o = 16; o >= CH; o >>= 1)
+            for (int i = 0; i < 8; ++i) v[i] += __shfl_xor_sync(0xffffffffu, v[i], o);
 #pragma unroll
-            for (int i = 0; i < CH; ++i) v[i] += __shfl_xor_sync(0xffffffffu, v[i], o);
-#pragma unroll
-        for (int k = CH / 2; k >= 1; k >>= 1) {
+        for (int k = 4; k >= 1; k >>= 1) {
             const bool up = (lane & k) != 0;
 #pragma unroll
             for (int i = 0; i < k; ++i) {
@@ -815,28 +871,27 @@ __device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& 
                 v[i] = (up ? v[i + k] : v[i]) + recv;
             }
         }
-        if (lane < CH) cx.lred[q4 * 128 + col0 + ch * CH + lane] = v[0];
+        if (lane < 8) cx.lred[q4 * 128 + col0 + ch * 8 + lane] = v[0];
     }
     soft_sync();
     const int pair = sg.s * p.hkv + sg.g;
     const int slot = blockIdx.x + pair;
     const bool whole = sg.j0 == 0 && sg.j1 == sg.nt;       // this CTA saw every tile of the pair
-    const uint32_t o_addr = cx.tmem + lane_base + TM_O + col0;
     if (p.pair_cnt && whole) {
         // no other partial exists: normalise and write the output directly
-        if (tid < NP) cx.alpha[tid] = 1.f / ((cx.lred[tid] + cx.lred[128 + tid]) + (cx.lred[256 + tid] + cx.lred[384 + tid]));
+        if (tid < np) cx.alpha[tid] = 1.f / ((cx.lred[tid] + cx.lred[128 + tid]) + (cx.lred[256 + tid] + cx.lred[384 + tid]));
         soft_sync();
         if (!dead) {
             __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(p.out);
-#pragma unroll
-            for (int ch = 0; ch < NCH; ++ch) {
-                uint32_t ov[CH];
-                tmem_ld<CH>(o_addr + ch * CH, ov);
+#pragma unroll 1
+            for (int ch = 0; ch < nch; ++ch) {
+                uint32_t ov[8];
+                tmem_ld<8>(o_addr + ch * 8, ov);
                 tmem_wait_ld();
-                int b = (col0 + ch * CH) / G, hg = (col0 + ch * CH) - b * G;
+                int b = (col0 + ch * 8) / G, hg = (col0 + ch * 8) - b * G;
 #pragma unroll
-                for (int i = 0; i < CH; ++i) {
-                    const int n = col0 + ch * CH + i;
+                for (int i = 0; i < 8; ++i) {
+                    const int n = col0 + ch * 8 + i;
                     if (n < M)
                         out[(((size_t)sg.s * p.max_active + b) * p.hq + (size_t)sg.g * G + hg) * D + krow] =
                             __float2bfloat16_rn(__uint_as_float(ov[i]) * cx.alpha[n]);
@@ -856,14 +911,14 @@ __device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& 
             }
             // O^T: lane = head_dim index, column = query row; partials are stored [query row][head_dim]
             float* wo = p.ws_o + (size_t)slot * p.mmax * D + krow;
-#pragma unroll
-            for (int ch = 0; ch < NCH; ++ch) {
-                uint32_t ov[CH];
-                tmem_ld<CH>(o_addr + ch * CH, ov);
+#pragma unroll 1
+            for (int ch = 0; ch < nch; ++ch) {
+                uint32_t ov[8];
+                tmem_ld<8>(o_addr + ch * 8, ov);
                 tmem_wait_ld();
 #pragma unroll
-                for (int i = 0; i < CH; ++i)
-                    if (col0 + ch * CH + i < M) wo[(size_t)(col0 + ch * CH + i) * D] = __uint_as_float(ov[i]);
+                for (int i = 0; i < 8; ++i)
+                    if (col0 + ch * 8 + i < M) wo[(size_t)(col0 + ch * 8 + i) * D] = __uint_as_float(ov[i]);
             }
         }
         if (p.pair_cnt) {
@@ -880,70 +935,9 @@ __device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& 
                 if (old == expected - 1) p.pair_cnt[pair] = 0;          // ready for the next call
             }
             soft_sync();
-            if (cx.flags[1]) {
-                __threadfence();
-                const int c_first = cx.flags[2], c_last = cx.flags[3];
-                // one thread per query row: m = max_c m_c, l = sum_c l_c 2^(m_c - m); the weight
-                // 2^(m_c - m) / l of every partial replaces m_c in the workspace.  Loads are issued
-                // four at a time: each costs a trip to L2 and nothing depends on the previous one.
-                if (tid < M) {
-                    float* ml = p.ws_ml + ((size_t)pair * p.mmax + tid) * 2;
-                    const size_t cs = (size_t)p.mmax * 2;                // stride between CTAs' entries
-                    float mx = -INFINITY;
-                    for (int c0 = c_first; c0 <= c_last; c0 += 4) {
-                        float v[4];
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) v[j] = c0 + j <= c_last ? __ldcg(ml + (size_t)(c0 + j) * cs) : -INFINITY;
-                        mx = fmaxf(fmaxf(mx, fmaxf(v[0], v[1])), fmaxf(v[2], v[3]));
-                    }
-                    float lt = 0.f;
-                    for (int c0 = c_first; c0 <= c_last; c0 += 4) {
-                        float2 v[4];
-#pragma unroll
-                        for (int j = 0; j < 4; ++j)
-                            v[j] = c0 + j <= c_last ? __ldcg(reinterpret_cast<const float2*>(ml + (size_t)(c0 + j) * cs)) : make_float2(-INFINITY, 0.f);
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) lt = fmaf(v[j].y, fast_exp2(v[j].x - mx), lt);   // a split that saw nothing: -inf -> 0
-                    }
-                    const float inv = 1.f / lt;
-                    for (int c = c_first; c <= c_last; ++c) {
-                        const float w = fast_exp2(__ldcg(ml + (size_t)c * cs) - mx) * inv;
-                        __stcg(ml + (size_t)c * cs, w);
-                    }
-                }
-                __threadfence();
-                soft_sync();
-                __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(p.out);
-                for (int idx = tid; idx < M * (D / 4); idx += NSOFT * 32) {
-                    const int m = idx / (D / 4), c4 = idx - m * (D / 4);
-                    const float* ml = p.ws_ml + ((size_t)pair * p.mmax + m) * 2;
-                    const float4* po = reinterpret_cast<const float4*>(p.ws_o + ((size_t)pair * p.mmax + m) * D) + c4;
-                    const size_t cs = (size_t)p.mmax * 2, os = (size_t)p.mmax * (D / 4);
-                    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-                    for (int c0 = c_first; c0 <= c_last; c0 += 4) {
-                        float w[4];
-                        float4 o[4];
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            const bool on = c0 + j <= c_last;
-                            w[j] = on ? __ldcg(ml + (size_t)(c0 + j) * cs) : 0.f;
-                            o[j] = on ? __ldcg(po + (size_t)(c0 + j) * os) : make_float4(0.f, 0.f, 0.f, 0.f);
-                        }
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            acc.x = fmaf(o[j].x, w[j], acc.x);
-                            acc.y = fmaf(o[j].y, w[j], acc.y);
-                            acc.z = fmaf(o[j].z, w[j], acc.z);
-                            acc.w = fmaf(o[j].w, w[j], acc.w);
-                        }
-                    }
-                    const int b = m / G, hg = m - b * G;
-                    uint2 pk;
-                    pk.x = pack2(acc.x, acc.y);
-                    pk.y = pack2(acc.z, acc.w);
-                    *reinterpret_cast<uint2*>(out + (((size_t)sg.s * p.max_active + b) * p.hq + (size_t)sg.g * G + hg) * D + c4 * 4) = pk;
-                }
-            }
+            if (cx.flags[1])
+                merge_pair(p.ws_ml, p.ws_o, reinterpret_cast<__nv_bfloat16*>(p.out), pair, p.mmax, M, G, sg.s, sg.g, p.max_active, p.hq,
+                           cx.flags[2], cx.flags[3]);
         }
     }
     soft_sync();                     // column state and Q^T are free again
@@ -952,10 +946,6 @@ __device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& 
     if (!dead && lane == 0) mbar_arrive(cx.o_free);
 }
 
-// NPMAX = query rows per (scene, KV head) the launch can meet, rounded up to 16/32/64/128: only
-// the softmax variants that can occur are compiled into a kernel, which keeps the register
-// allocation of the narrow ones free of the wide ones' pressure.
-template <int NPMAX>
 __global__ void __launch_bounds__(THREADS, 1)
 attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
                const int nk, const int nv, const int np_max, const int npb)
@@ -1090,15 +1080,7 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, con
         while (u < hi) {
             const Segment sg = decode_segment(u, hi, cx.pre, p.hkv, s);
             const int M = cx.nact[sg.s] * p.group;
-            if (NPMAX == 16 || M <= 16) {
-                softmax_segment<8>(p, cx, sg, seg, hi, prefetched, g, dead, warp, lane);
-            } else if (NPMAX == 32 || M <= 32) {
-                if constexpr (NPMAX >= 32) softmax_segment<16>(p, cx, sg, seg, hi, prefetched, g, dead, warp, lane);
-            } else if (NPMAX == 64 || M <= 64) {
-                if constexpr (NPMAX >= 64) softmax_segment<32>(p, cx, sg, seg, hi, prefetched, g, dead, warp, lane);
-            } else {
-                if constexpr (NPMAX >= 128) softmax_segment<64>(p, cx, sg, seg, hi, prefetched, g, dead, warp, lane);
-            }
+            softmax_segment(p, cx, sg, M <= 16 ? 8 : (M <= 32 ? 16 : (M <= 64 ? 32 : 64)), seg, hi, prefetched, g, dead, warp, lane);
             ++seg;
             u = sg.next_u;
         }
@@ -1136,21 +1118,13 @@ int launch_attn_tc(const AttnParams& p, int head_dim, cudaStream_t st)
     if (rc) return rc;
     rc = get_kv_tensor_map(p.v, p, D, TILE, &tv);
     if (rc) return rc;
-    auto launch = [&](auto kernel, size_t& attr_smem) -> int {
-        if (smem > attr_smem) {
-            cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-            if (e != cudaSuccess) return set_cuda_error(e);
-            attr_smem = smem;
-        }
-        kernel<<<p.n_cta, THREADS, smem, st>>>(p, tk, tv, nk, nv, np_max, npb);
-        return FDC_OK;
-    };
-    static size_t attr16 = 0, attr32 = 0, attr64 = 0, attr128 = 0;
-    if (np_max == 16) rc = launch(attn_tc_kernel<16>, attr16);
-    else if (np_max == 32) rc = launch(attn_tc_kernel<32>, attr32);
-    else if (np_max == 64) rc = launch(attn_tc_kernel<64>, attr64);
-    else rc = launch(attn_tc_kernel<128>, attr128);
-    if (rc) return rc;
+    static size_t attr_smem = 0;
+    if (smem > attr_smem) {
+        cudaError_t e = cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return set_cuda_error(e);
+        attr_smem = smem;
+    }
+    attn_tc_kernel<<<p.n_cta, THREADS, smem, st>>>(p, tk, tv, nk, nv, np_max, npb);
     note_launch();
     cudaError_t e = cudaGetLastError();
     return e == cudaSuccess ? FDC_OK : set_cuda_error(e);
