@@ -6,17 +6,17 @@
 // work scales with the real number of queries and every TMEM lane / softmax thread owns a
 // real KV row:
 //     S^T = K Q^T      M = 128 KV rows (one "round" = two 64-row tiles of the visited-tile
-//                      list), N = NP query rows (16/32/64/128), K = head_dim;  A = the K tiles
+//                      list), N = NP query rows (32/64/128), K = head_dim;  A = the K tiles
 //                      as TMA left them in shared memory, B = Q^T staged once per segment
 //     O^T += V^T P^T   M = head_dim, N = NP, K = 128 KV rows;  A = the V tiles (M-major), B =
 //                      P^T written by the softmax threads (N-major), accumulator in TMEM
 // One persistent CTA per SM:
-//   warps 8, 10  TMA producers: K stages and V stages (128 rows, 128B swizzle) of two rings
-//   warp 9       issues S^T = K Q^T (one elected thread); allocates / frees TMEM.  S^T is double
+//   warps 16, 18 TMA producers: K stages and V stages (128 rows, 128B swizzle) of two rings
+//   warp 17      issues S^T = K Q^T (one elected thread); allocates / frees TMEM.  S^T is double
 //                buffered in TMEM, so K Q^T of round r+1 overlaps the softmax of round r
-//   warp 11      clears the V rows that no branch may see (they can hold anything, NaN included,
+//   warp 19      clears the V rows that no branch may see (they can hold anything, NaN included,
 //                and 0 * NaN must not reach the accumulator), then issues O^T += V^T P^T
-//   warps 0-7    softmax.  Thread = one KV row of the round (TMEM lane) x half of the query
+//   warps 0-15   softmax.  Thread = one KV row of the round (TMEM lane) x a quarter of the query
 //                columns.  Eq. 1 is applied by select from the branches' row bitmaps; prefix
 //                tiles skip it.
 // The softmax reference of a query column is raised lazily: it is set from the column maximum
@@ -37,9 +37,10 @@ namespace {
 constexpr int D = 128;                       // head_dim handled by this kernel
 constexpr int TILE = FDC_TILE_ROWS;          // rows per entry of the visited-tile list
 constexpr int RROWS = 2 * TILE;              // KV rows per round = M of S^T = K of O^T
-constexpr int NSOFT = 8;                     // softmax warps
-constexpr int W_KPROD = 8, W_QK = 9, W_VPROD = 10, W_PV = 11;
-constexpr int THREADS = 384;
+constexpr int NSOFT = 16;                    // softmax warps: 4 row quadrants x 4 column parts
+constexpr int NPART = NSOFT / 4;             // column parts
+constexpr int W_KPROD = NSOFT, W_QK = NSOFT + 1, W_VPROD = NSOFT + 2, W_PV = NSOFT + 3;
+constexpr int THREADS = (NSOFT + 4) * 32;
 constexpr uint32_t TMEM_COLS = 512;          // S^T 0 [0,128) | S^T 1 [128,256) | O^T [256,384) | sums [384,512)
 constexpr uint32_t TM_O = 256;
 constexpr uint32_t TM_L = 384;                // per-column sums of the softmax threads [384, 512)
@@ -311,7 +312,7 @@ __device__ __forceinline__ void qk_loop(const AttnParams& p, const Ctx& cx, long
         const int nr = (sg.j1 - sg.j0 + 1) >> 1;
         if (lane == 0) {
             const int M = cx.nact[sg.s] * p.group;
-            const int NP = M <= 16 ? 16 : (M <= 32 ? 32 : (M <= 64 ? 64 : 128));
+            const int NP = M <= 32 ? 32 : (M <= 64 ? 64 : 128);
             const uint32_t idesc_qk = instr_desc(RROWS, NP, 0);
             bool good = mbar_wait(cx.q_ready, seg & 1, cx.abortp, p.status);
             for (int t = 0; t < nr && good; ++t, ++g) {
@@ -362,7 +363,7 @@ __device__ __forceinline__ void pv_loop(const AttnParams& p, const Ctx& cx, long
         const Segment sg = decode_segment(u, hi, cx.pre, p.hkv, s);
         const int A = cx.nact[sg.s];
         const int M = A * p.group;
-        const int NP = M <= 16 ? 16 : (M <= 32 ? 32 : (M <= 64 ? 64 : 128));
+        const int NP = M <= 32 ? 32 : (M <= 64 ? 64 : 128);
         const uint32_t idesc_pv = instr_desc(D, NP, 1);
         if (cx.mstaged) {                            // the softmax warps publish the scene's bitmaps with the queries
             int okw = 1;
@@ -480,7 +481,7 @@ __device__ __noinline__ void prefetch_next_segment(const uint4* qg, const uint64
     int s2 = s_cur;
     const Segment nx = decode_segment(next_u, hi, pre, hkv, s2);
     const int M2 = nact[nx.s] * G;
-    const int NP2 = M2 <= 16 ? 16 : (M2 <= 32 ? 32 : (M2 <= 64 ? 64 : 128));
+    const int NP2 = M2 <= 32 ? 32 : (M2 <= 64 ? 64 : 128);
     for (int idx = tid; idx < NP2 * (D / 8); idx += NSOFT * 32) {
         const int n = idx / (D / 8), ch = idx - n * (D / 8);
         const bool valid = n < M2;
@@ -581,7 +582,7 @@ struct RaiseArgs {
 };
 __device__ __noinline__ int raise_references(const RaiseArgs a)
 {
-    const int np = 2 * a.nph;
+    const int np = NPART * a.nph;
     float* alpha = a.mneg + 128;
     int* wmax = reinterpret_cast<int*>(a.mneg + 256);      // [4][128]: maxima per row quadrant (shares the lred block)
     int* flags = reinterpret_cast<int*>(a.mneg + 768) + 128;
@@ -673,19 +674,19 @@ __device__ __noinline__ int raise_references(const RaiseArgs a)
     return dead ? 1 : 0;
 }
 
-// The softmax warps' work on one segment; nph = query columns per thread (half of NP: 8, 16, 32
-// or 64).  Columns are handled eight at a time in real loops, with the per-column sums kept in
+// The softmax warps' work on one segment; nph = query columns per thread (a quarter of NP: 8, 16
+// or 32).  Columns are handled eight at a time in real loops, with the per-column sums kept in
 // TMEM (the free columns [384, 512)) and the references read from shared memory, so that the
 // same small loop serves every width.
 __device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& cx, const Segment& sg, const int nph, const uint32_t seg,
                                                 const long long hi, int& prefetched, uint32_t& g, bool& dead, const int warp, const int lane)
 {
-    const int np = 2 * nph, nch = nph >> 3;
-    const int tid = threadIdx.x;                  // 0..255
-    const int q4 = warp & 3, half = warp >> 2;
+    const int np = NPART * nph, nch = nph >> 3;
+    const int tid = threadIdx.x;                  // 0..NSOFT * 32 - 1
+    const int q4 = warp & 3, part = warp >> 2;
     const int krow = q4 * 32 + lane;              // KV row of the round = TMEM lane of S^T; head_dim index for O^T
     const uint32_t lane_base = (uint32_t)(q4 * 32) << 16;
-    const int col0 = half * nph;
+    const int col0 = part * nph;
     const float c = p.scale_log2;
     const int A = cx.nact[sg.s];
     const int M = A * p.group;
@@ -706,9 +707,10 @@ __device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& 
         } else {
             // all global reads first (one latency), then the stores
             const uint4* qg = reinterpret_cast<const uint4*>(p.q);
-            uint4 qv[8];
+            constexpr int QPT = 128 * (D / 8) / (NSOFT * 32);      // 16-byte chunks per thread for 128 query rows
+            uint4 qv[QPT];
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
+            for (int i = 0; i < QPT; ++i) {
                 const int idx = tid + i * (NSOFT * 32);
                 const int n = idx / (D / 8), ch = idx - n * (D / 8);
                 qv[i] = make_uint4(0u, 0u, 0u, 0u);
@@ -725,7 +727,7 @@ __device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& 
                 mv[i] = idx < nw ? p.mask[(size_t)sg.s * p.max_active * p.W + idx] : 0ull;
             }
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
+            for (int i = 0; i < QPT; ++i) {
                 const int idx = tid + i * (NSOFT * 32);
                 const int n = idx / (D / 8), ch = idx - n * (D / 8);
                 if (n < np) *reinterpret_cast<uint4*>(cx.qs + (ch >> 3) * cx.q_panel + n * 128 + (((ch & 7) ^ (n & 7)) << 4)) = qv[i];
@@ -1080,7 +1082,7 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, con
         while (u < hi) {
             const Segment sg = decode_segment(u, hi, cx.pre, p.hkv, s);
             const int M = cx.nact[sg.s] * p.group;
-            softmax_segment(p, cx, sg, M <= 16 ? 8 : (M <= 32 ? 16 : (M <= 64 ? 32 : 64)), seg, hi, prefetched, g, dead, warp, lane);
+            softmax_segment(p, cx, sg, (M <= 32 ? 32 : (M <= 64 ? 64 : 128)) / NPART, seg, hi, prefetched, g, dead, warp, lane);
             ++seg;
             u = sg.next_u;
         }
@@ -1103,7 +1105,7 @@ namespace fdc {
 int launch_attn_tc(const AttnParams& p, int head_dim, cudaStream_t st)
 {
     if (head_dim != D || p.mmax > 128) return FDC_ERR_SHAPE;
-    const int np_max = p.mmax <= 16 ? 16 : (p.mmax <= 32 ? 32 : (p.mmax <= 64 ? 64 : 128));
+    const int np_max = p.mmax <= 32 ? 32 : (p.mmax <= 64 ? 64 : 128);
     const int p_buf = ((np_max + 63) / 64) * PANEL;
     const int npb = np_max > 64 ? 1 : 2;          // 128 query rows: one P^T buffer, so that four stages still fit
     const size_t fixed = 1024 + (size_t)npb * p_buf + (size_t)(D / 64) * np_max * 128 + 8 * (4 * MAXST + 8) + 16 +
