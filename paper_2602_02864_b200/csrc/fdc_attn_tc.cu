@@ -165,7 +165,8 @@ __device__ __forceinline__ float ord_to(int i) { return __int_as_float(i ^ ((i >
 
 // Everything a role needs to find its barriers and buffers.
 struct Ctx {
-    uint32_t k_full, k_empty, v_full, v_empty, s_full, p_full, pv_done, q_ready, o_free;
+    uint32_t k_full, k_empty, v_full, v_empty, s_full, s_free, p_full, pv_done, q_ready, o_free;
+    int ns, s_stride;                // S^T buffers in TMEM (4 of 64 columns up to 64 query rows, else 2 of 128) and their distance
     uint32_t tmem;
     unsigned char *kring, *vring, *qs, *ps;
     float *mneg, *alpha, *lred;      // [128] -reference per column, [128] rescale factors, [4][128] partial sums
@@ -294,8 +295,9 @@ __device__ __forceinline__ void producer_loop(const AttnParams& p, const Ctx& cx
     }
 }
 
-// Warp 9 (one elected thread): S^T[g & 1] = K(stage) Q^T for every round g.  The score buffer is
-// free again once the softmax threads have consumed round g - 2, which they signal with p_full.
+// One elected thread: S^T[g mod ns] = K(stage) Q^T for every round g.  A score buffer is free again
+// once the softmax threads have read round g - ns (s_free); with four buffers K Q^T runs well ahead of
+// the softmax, so a K stage is released soon after it landed and the K ring stays in flight.
 __device__ __forceinline__ void qk_loop(const AttnParams& p, const Ctx& cx, long long lo, long long hi, int lane)
 {
     const uint64_t q_desc = smem_desc(smem_u32(cx.qs), 16, 1024);
@@ -317,17 +319,18 @@ __device__ __forceinline__ void qk_loop(const AttnParams& p, const Ctx& cx, long
             bool good = mbar_wait(cx.q_ready, seg & 1, cx.abortp, p.status);
             for (int t = 0; t < nr && good; ++t, ++g) {
                 good = mbar_wait(cx.k_full + 8 * st, kph, cx.abortp, p.status);
-                if (good && g >= 2) good = mbar_wait(cx.p_full + 8 * (g & 1), ((g - 2) >> 1) & 1, cx.abortp, p.status);
+                const uint32_t sb = g & (cx.ns - 1);                  // score buffer of the round
+                if (good && g >= (uint32_t)cx.ns) good = mbar_wait(cx.s_free + 8 * sb, ((g / cx.ns) - 1) & 1, cx.abortp, p.status);
                 if (!good) break;
                 tc_fence_after();
                 const uint64_t kd = k_desc0 + (uint64_t)((st * STAGE) >> 4);
-                const uint32_t d = cx.tmem + (g & 1) * 128;
+                const uint32_t d = cx.tmem + sb * cx.s_stride;
 #pragma unroll
                 for (int ks = 0; ks < D / 16; ++ks)
                     umma(d, kd + (uint64_t)(((ks >> 2) * PANEL + (ks & 3) * 32) >> 4), q_desc + (ks >> 2) * qp16 + (uint64_t)(((ks & 3) * 32) >> 4),
                          idesc_qk, ks > 0);
                 umma_commit(cx.k_empty + 8 * st);
-                umma_commit(cx.s_full + 8 * (g & 1));
+                umma_commit(cx.s_full + 8 * sb);
                 if (++st == cx.nk) {
                     st = 0;
                     kph ^= 1;
@@ -766,7 +769,8 @@ __device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& 
             const bool masked = live && tile * TILE + TILE > p.P;
             // Eq. 1 for this thread's KV row: bit i of vis <=> column col0 + i may see the row
             const uint64_t vis = masked ? row_visibility(mask_row(p, cx, seg, sg.s, 0), p.W, p.P, tile, A, G, col0, nph, q4 & 1) : ~0ull;
-            wait_u(cx.s_full + 8 * b, (g >> 1) & 1);
+            const uint32_t sb = g & (cx.ns - 1);                      // score buffer of the round
+            wait_u(cx.s_full + 8 * sb, (g / cx.ns) & 1);
             tc_fence_after();
             if (jb + k + 2 >= ntile && sg.next_u < hi && !dead) {
                 // last round: every S^T = K Q^T of this segment has completed, so Q^T may be overwritten.
@@ -781,7 +785,7 @@ __device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& 
             // warp has also finished round g - 2, so what that round left in rflag is the same for all.
             if (cx.npb == 2) wait_u(cx.pv_done + 8 * b, ((g >> 1) & 1) ^ 1);
             else if (g > 0) wait_u(cx.pv_done + 8 * ((g - 1) & 1), ((g - 1) >> 1) & 1);
-            const uint32_t s_addr = cx.tmem + lane_base + b * 128 + col0;
+            const uint32_t s_addr = cx.tmem + lane_base + sb * cx.s_stride + col0;
             // References are set in the first round of a segment.  Later a score more than 2^16 above its
             // reference only leaves a note (no barrier in the common path): p stays far from overflow, and
             // two rounds later, when all warps are known to see the note, the references are raised.
@@ -844,7 +848,10 @@ __device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& 
             tc_fence_before();
             fence_async_smem();
             __syncwarp();
-            if (!dead && lane == 0) mbar_arrive(cx.p_full + 8 * b);
+            if (!dead && lane == 0) {
+                mbar_arrive(cx.s_free + 8 * sb);                       // the scores have been read: K Q^T may reuse the buffer
+                mbar_arrive(cx.p_full + 8 * b);
+            }
         }
     }
     // ---- end of segment: the accumulator is final once the last PV has completed
@@ -970,11 +977,14 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, con
     cx.v_full = cx.k_empty + 8 * MAXST;
     cx.v_empty = cx.v_full + 8 * MAXST;
     cx.s_full = cx.v_empty + 8 * MAXST;
-    cx.p_full = cx.s_full + 16;
+    cx.s_free = cx.s_full + 8 * 4;
+    cx.p_full = cx.s_free + 8 * 4;
+    cx.ns = np_max <= 64 ? 4 : 2;
+    cx.s_stride = np_max <= 64 ? 64 : 128;
     cx.pv_done = cx.p_full + 16;
     cx.q_ready = cx.pv_done + 16;
     cx.o_free = cx.q_ready + 8;
-    uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bars + 4 * MAXST + 8);
+    uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bars + 4 * MAXST + 14);
     cx.mneg = reinterpret_cast<float*>(tmem_holder + 4);
     cx.alpha = cx.mneg + 128;
     cx.lred = cx.alpha + 128;
@@ -1044,8 +1054,11 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, con
             mbar_init(cx.v_full + 8 * i, 1);
             mbar_init(cx.v_empty + 8 * i, 1);
         }
-        for (int i = 0; i < 2; ++i) {
+        for (int i = 0; i < 4; ++i) {
             mbar_init(cx.s_full + 8 * i, 1);
+            mbar_init(cx.s_free + 8 * i, NSOFT);
+        }
+        for (int i = 0; i < 2; ++i) {
             mbar_init(cx.p_full + 8 * i, NSOFT);
             mbar_init(cx.pv_done + 8 * i, 1);
         }
@@ -1108,7 +1121,7 @@ int launch_attn_tc(const AttnParams& p, int head_dim, cudaStream_t st)
     const int np_max = p.mmax <= 32 ? 32 : (p.mmax <= 64 ? 64 : 128);
     const int p_buf = ((np_max + 63) / 64) * PANEL;
     const int npb = np_max > 64 ? 1 : 2;          // 128 query rows: one P^T buffer, so that four stages still fit
-    const size_t fixed = 1024 + (size_t)npb * p_buf + (size_t)(D / 64) * np_max * 128 + 8 * (4 * MAXST + 8) + 16 +
+    const size_t fixed = 1024 + (size_t)npb * p_buf + (size_t)(D / 64) * np_max * 128 + 8 * (4 * MAXST + 14) + 16 +
                          4 * (128 + 128 + 512 + 128 + 8) + sizeof(int) * (3 * p.batch + 2) + 8 * (2 * MBUF + 2) + 64;
     int stages = (int)((227 * 1024 - 256 - fixed) / STAGE);
     if (stages > 2 * MAXST) stages = 2 * MAXST;
