@@ -89,6 +89,17 @@ __device__ __forceinline__ void umma(uint32_t d_tmem, uint64_t a_desc, uint64_t 
         ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
         : "memory");
 }
+// The same with the descriptors given as (low, high) words: the address field sits in the low
+// word, so stepping through an operand is 32-bit arithmetic for the issuing thread.
+__device__ __forceinline__ void umma2(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi, uint32_t idesc,
+                                      uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\tsetp.ne.b32 p, %6, 0;\n\tmov.b64 da, {%1, %2};\n\tmov.b64 db, {%3, %4};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %5, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
 __device__ __forceinline__ void umma_commit(uint32_t bar)
 {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
@@ -302,7 +313,8 @@ __device__ __forceinline__ void qk_loop(const AttnParams& p, const Ctx& cx, long
 {
     const uint64_t q_desc = smem_desc(smem_u32(cx.qs), 16, 1024);
     const uint64_t k_desc0 = smem_desc(smem_u32(cx.kring), 16, 1024);
-    const uint64_t qp16 = (uint64_t)(cx.q_panel >> 4);
+    const uint32_t q_lo = (uint32_t)q_desc, q_hi = (uint32_t)(q_desc >> 32), k_lo0 = (uint32_t)k_desc0, k_hi = (uint32_t)(k_desc0 >> 32);
+    const uint32_t qp16 = (uint32_t)(cx.q_panel >> 4);
     int s = 0;
     uint32_t g = 0, seg = 0;
     int st = 0;
@@ -323,12 +335,12 @@ __device__ __forceinline__ void qk_loop(const AttnParams& p, const Ctx& cx, long
                 if (good && g >= (uint32_t)cx.ns) good = mbar_wait(cx.s_free + 8 * sb, ((g / cx.ns) - 1) & 1, cx.abortp, p.status);
                 if (!good) break;
                 tc_fence_after();
-                const uint64_t kd = k_desc0 + (uint64_t)((st * STAGE) >> 4);
+                const uint32_t kd = k_lo0 + (uint32_t)((st * STAGE) >> 4);
                 const uint32_t d = cx.tmem + sb * cx.s_stride;
 #pragma unroll
                 for (int ks = 0; ks < D / 16; ++ks)
-                    umma(d, kd + (uint64_t)(((ks >> 2) * PANEL + (ks & 3) * 32) >> 4), q_desc + (ks >> 2) * qp16 + (uint64_t)(((ks & 3) * 32) >> 4),
-                         idesc_qk, ks > 0);
+                    umma2(d, kd + (uint32_t)(((ks >> 2) * PANEL + (ks & 3) * 32) >> 4), k_hi, q_lo + (ks >> 2) * qp16 + (uint32_t)(((ks & 3) * 32) >> 4), q_hi,
+                          idesc_qk, ks > 0);
                 umma_commit(cx.k_empty + 8 * st);
                 umma_commit(cx.s_full + 8 * sb);
                 if (++st == cx.nk) {
@@ -347,6 +359,43 @@ __device__ __forceinline__ void qk_loop(const AttnParams& p, const Ctx& cx, long
     }
 }
 
+// V rows of a stage that are invisible to every branch of the scene are cleared (whole warp; kept
+// out of line: only rounds beyond the prefix come here).  tile0 / tile1 are the round's tiles.
+__device__ __noinline__ void clear_unseen_rows(unsigned char* vs, const uint64_t* mask0, int W, int P, int A, int tile0, int tile1, int nt)
+{
+    const int lane = threadIdx.x & 31;
+    bool touched = false;
+    for (int i = 0; i < nt; ++i) {
+        const int tile = i ? tile1 : tile0;
+        if (tile * TILE + TILE <= P) continue;                 // all rows visible to everybody
+        uint64_t um = 0ull;
+        for (int b = lane; b < A; b += 32) um |= tile_rowmask(mask0 + (size_t)b * W, W, P, tile);
+        const uint32_t ul = __reduce_or_sync(0xffffffffu, (uint32_t)um);
+        const uint32_t uh = __reduce_or_sync(0xffffffffu, (uint32_t)(um >> 32));
+        const uint64_t z = ~(((uint64_t)uh << 32) | ul);
+        if (z) {
+            // lane l clears rows l and l + 32 of the tile if nobody sees them (2 panels x 8 chunks of 16 bytes)
+#pragma unroll
+            for (int hr = 0; hr < 2; ++hr) {
+                const int r = lane + 32 * hr;
+                if ((z >> r) & 1) {
+                    unsigned char* row = vs + (i * TILE + r) * 128;
+#pragma unroll
+                    for (int ch = 0; ch < 8; ++ch) {
+                        // rotate the chunk order by the row so that the lanes of a warp hit different banks
+                        const int cc = ((ch + r) & 7) << 4;
+                        *reinterpret_cast<uint4*>(row + cc) = make_uint4(0u, 0u, 0u, 0u);
+                        *reinterpret_cast<uint4*>(row + PANEL + cc) = make_uint4(0u, 0u, 0u, 0u);
+                    }
+                }
+            }
+            touched = true;
+        }
+    }
+    if (touched) fence_async_smem();
+    __syncwarp();
+}
+
 // Warp 11: O^T += V^T(stage) P^T[g & 1] for every round g (one elected thread issues).  Before
 // that the whole warp clears the V rows of the stage that are invisible to every branch of the
 // scene: their P^T row is exactly 0, but the rows can hold anything (NaN, Inf) and 0 * NaN must
@@ -355,6 +404,7 @@ __device__ __forceinline__ void pv_loop(const AttnParams& p, const Ctx& cx, long
 {
     const uint64_t v_desc0 = smem_desc(smem_u32(cx.vring), PANEL, 1024);
     const uint64_t p_desc0 = smem_desc(smem_u32(cx.ps), PANEL, 1024);
+    const uint32_t v_lo0 = (uint32_t)v_desc0, v_hi = (uint32_t)(v_desc0 >> 32), p_lo0 = (uint32_t)p_desc0, p_hi = (uint32_t)(p_desc0 >> 32);
     const uint32_t tm_o = cx.tmem + TM_O;
     int s = 0;
     uint32_t g = 0, seg = 0;
@@ -379,56 +429,28 @@ __device__ __forceinline__ void pv_loop(const AttnParams& p, const Ctx& cx, long
             const int my_tile = lane < jn ? p.tiles[(size_t)sg.s * p.ntile_max + jb + lane] : 0;
             for (int k = 0; k < jn && ok; k += 2, ++g, ++t) {
                 const int nt = jn - k < 2 ? 1 : 2;
+                // tile ids ascend: the round reaches beyond the prefix iff its last tile does
+                const int t_last = __shfl_sync(0xffffffffu, my_tile, (k + nt - 1) & 31);
                 int okw = 1;
                 if (lane == 0) okw = mbar_wait(cx.v_full + 8 * st, vph, cx.abortp, p.status);
-                ok = __shfl_sync(0xffffffffu, okw, 0);
-                if (!ok) break;
-                unsigned char* vs = cx.vring + (size_t)st * STAGE;
-                bool touched = false;
-                for (int i = 0; i < nt; ++i) {
-                    const int tile = __shfl_sync(0xffffffffu, my_tile, (k + i) & 31);
-                    if (tile * TILE + TILE <= p.P) continue;                 // all rows visible to everybody
-                    uint64_t um = 0ull;
-                    for (int b = lane; b < A; b += 32)
-                        um |= tile_rowmask(mask_row(p, cx, seg, sg.s, b), p.W, p.P, tile);
-                    const uint32_t ul = __reduce_or_sync(0xffffffffu, (uint32_t)um);
-                    const uint32_t uh = __reduce_or_sync(0xffffffffu, (uint32_t)(um >> 32));
-                    const uint64_t z = ~(((uint64_t)uh << 32) | ul);
-                    if (z) {
-                        // lane l clears rows l and l + 32 of the tile if nobody sees them (2 panels x 8 chunks of 16 bytes)
-#pragma unroll
-                        for (int hr = 0; hr < 2; ++hr) {
-                            const int r = lane + 32 * hr;
-                            if ((z >> r) & 1) {
-                                unsigned char* row = vs + (i * TILE + r) * 128;
-#pragma unroll
-                                for (int ch = 0; ch < 8; ++ch) {
-                                    // rotate the chunk order by the row so that the lanes of a warp hit different banks
-                                    const int cc = ((ch + r) & 7) << 4;
-                                    *reinterpret_cast<uint4*>(row + cc) = make_uint4(0u, 0u, 0u, 0u);
-                                    *reinterpret_cast<uint4*>(row + PANEL + cc) = make_uint4(0u, 0u, 0u, 0u);
-                                }
-                            }
-                        }
-                        touched = true;
-                    }
+                if (t_last * TILE + TILE > p.P) {
+                    okw = __shfl_sync(0xffffffffu, okw, 0);
+                    if (okw)
+                        clear_unseen_rows(cx.vring + (size_t)st * STAGE, mask_row(p, cx, seg, sg.s, 0), p.W, p.P, A,
+                                          __shfl_sync(0xffffffffu, my_tile, k & 31), t_last, nt);
                 }
-                if (touched) fence_async_smem();
-                __syncwarp();
-                if (lane == 0) {
+                if (lane == 0 && okw) {
                     bool good = mbar_wait(cx.p_full + 8 * (g & 1), (g >> 1) & 1, cx.abortp, p.status);
                     if (good && t == 0 && seg > 0) good = mbar_wait(cx.o_free, (seg - 1) & 1, cx.abortp, p.status);
                     if (good) {
                         tc_fence_after();
-                        const uint64_t vd = v_desc0 + (uint64_t)((st * STAGE) >> 4);
-                        const uint64_t pd = p_desc0 + (uint64_t)((((g & 1) & (cx.npb - 1)) * cx.p_buf) >> 4);
+                        const uint32_t vd = v_lo0 + (uint32_t)((st * STAGE) >> 4);
+                        const uint32_t pd = p_lo0 + (uint32_t)((((g & 1) & (cx.npb - 1)) * cx.p_buf) >> 4);
 #pragma unroll
-                        for (int kk = 0; kk < 4; ++kk)
-                            umma(tm_o, vd + (uint64_t)((kk * 2048) >> 4), pd + (uint64_t)((kk * 2048) >> 4), idesc_pv, (t > 0 || kk > 0) ? 1u : 0u);
+                        for (int kk = 0; kk < 4; ++kk) umma2(tm_o, vd + kk * 128, v_hi, pd + kk * 128, p_hi, idesc_pv, (t > 0 || kk > 0) ? 1u : 0u);
                         if (nt == 2) {                                       // a one-tile round has 64 KV rows
 #pragma unroll
-                            for (int kk = 4; kk < 8; ++kk)
-                                umma(tm_o, vd + (uint64_t)((kk * 2048) >> 4), pd + (uint64_t)((kk * 2048) >> 4), idesc_pv, 1u);
+                            for (int kk = 4; kk < 8; ++kk) umma2(tm_o, vd + kk * 128, v_hi, pd + kk * 128, p_hi, idesc_pv, 1u);
                         }
                         umma_commit(cx.v_empty + 8 * st);
                         umma_commit(cx.pv_done + 8 * (g & 1));
