@@ -1022,6 +1022,11 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, con
     cx.abortp = &abort_flag;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // Programmatic dependent launch: this grid may have been scheduled while the kernel before it in
+    // the stream was still running.  Nothing of global memory is touched before that kernel has
+    // completed; the kernel after this one may be scheduled early in the same way.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (threadIdx.x == 0) abort_flag = 0;
     if (threadIdx.x < 4) cx.rflag[threadIdx.x] = -1;
     for (int i = threadIdx.x; i < p.batch; i += THREADS) cx.nact[i] = p.n_active[i];
@@ -1161,7 +1166,20 @@ int launch_attn_tc(const AttnParams& p, int head_dim, cudaStream_t st)
         if (e != cudaSuccess) return set_cuda_error(e);
         attr_smem = smem;
     }
-    attn_tc_kernel<<<p.n_cta, THREADS, smem, st>>>(p, tk, tv, nk, nv, np_max, npb);
+    {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(p.n_cta);
+        cfg.blockDim = dim3(THREADS);
+        cfg.dynamicSmemBytes = smem;
+        cfg.stream = st;
+        cudaLaunchAttribute at[1];
+        at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        at[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = at;
+        cfg.numAttrs = 1;
+        cudaError_t e = cudaLaunchKernelEx(&cfg, attn_tc_kernel, p, tk, tv, nk, nv, np_max, npb);
+        if (e != cudaSuccess) return set_cuda_error(e);
+    }
     note_launch();
     cudaError_t e = cudaGetLastError();
     return e == cudaSuccess ? FDC_OK : set_cuda_error(e);

@@ -19,6 +19,10 @@ __global__ void kv_append_kernel(char* __restrict__ k, char* __restrict__ v, int
                                  const int32_t* __restrict__ kv_row, const char* __restrict__ k_new,
                                  const char* __restrict__ v_new, int32_t* __restrict__ status)
 {
+    // programmatic dependent launch (see the attention kernel): wait for the kernel before this one,
+    // let the one after it be scheduled
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int s = blockIdx.x / max_active, b = blockIdx.x - s * max_active;
     if (b >= n_active[s]) return;
     const int row = kv_row[blockIdx.x];
@@ -75,10 +79,21 @@ extern "C" int fdc_kv_append(const fdc_plan* p, const fdc_kv_desc* kv, int32_t l
     const int row_bytes = kv->head_dim * es;
     int threads = kv->hkv * (row_bytes >> 4);
     threads = threads > 256 ? 256 : ((threads + 31) & ~31);
-    kv_append_kernel<<<kv->batch * p->h.max_active, threads, 0, (cudaStream_t)stream>>>(
-        kb, vb, kv->stride_scene * es, kv->stride_head * es, kv->stride_row * es, kv->rows, kv->hkv, row_bytes,
-        p->h.max_active, d_n_active, d_kv_row, (const char*)d_k_new, (const char*)d_v_new, p->d_status);
+    {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(kv->batch * p->h.max_active);
+        cfg.blockDim = dim3(threads);
+        cfg.dynamicSmemBytes = 0;
+        cfg.stream = (cudaStream_t)stream;
+        cudaLaunchAttribute at[1];
+        at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        at[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = at;
+        cfg.numAttrs = 1;
+        FDC_CUDA(cudaLaunchKernelEx(&cfg, kv_append_kernel, kb, vb, (int64_t)(kv->stride_scene * es), (int64_t)(kv->stride_head * es),
+                                    (int64_t)(kv->stride_row * es), (int)kv->rows, (int)kv->hkv, row_bytes, (int)p->h.max_active, d_n_active,
+                                    d_kv_row, (const char*)d_k_new, (const char*)d_v_new, p->d_status));
+    }
     note_launch();
-    FDC_CUDA(cudaGetLastError());
     return FDC_OK;
 }
