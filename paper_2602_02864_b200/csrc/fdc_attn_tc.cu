@@ -1022,26 +1022,59 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, con
     cx.abortp = &abort_flag;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) abort_flag = 0;
+    if (threadIdx.x < 4) cx.rflag[threadIdx.x] = -1;
+    // ---- set-up that needs no global memory: barriers, TMEM
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < MAXST; ++i) {
+            mbar_init(cx.k_full + 8 * i, 1);
+            mbar_init(cx.k_empty + 8 * i, 1);
+            mbar_init(cx.v_full + 8 * i, 1);
+            mbar_init(cx.v_empty + 8 * i, 1);
+        }
+        for (int i = 0; i < 4; ++i) {
+            mbar_init(cx.s_full + 8 * i, 1);
+            mbar_init(cx.s_free + 8 * i, NSOFT);
+        }
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(cx.p_full + 8 * i, NSOFT);
+            mbar_init(cx.pv_done + 8 * i, 1);
+        }
+        mbar_init(cx.q_ready, NSOFT);
+        mbar_init(cx.o_free, NSOFT);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        fence_async_smem();
+    }
+    if (warp == W_QK) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_holder)), "r"(TMEM_COLS)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *reinterpret_cast<volatile uint32_t*>(tmem_holder);
+    cx.tmem = tmem;
     // Programmatic dependent launch: this grid may have been scheduled while the kernel before it in
     // the stream was still running.  Nothing of global memory is touched before that kernel has
     // completed; the kernel after this one may be scheduled early in the same way.
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    if (threadIdx.x == 0) abort_flag = 0;
-    if (threadIdx.x < 4) cx.rflag[threadIdx.x] = -1;
+    bool active = true;                       // this CTA has units (uniform over the CTA)
+    long long lo = 0, hi = 0;
     for (int i = threadIdx.x; i < p.batch; i += THREADS) cx.nact[i] = p.n_active[i];
     const long long total = scan_ntiles(p.ntiles, p.batch, cx.pre);
     const long long U = total * p.hkv;
-    if (U == 0) return;
+    if (U == 0) active = false;
     // small problems use fewer CTAs (fewer partials to merge); every participating CTA owns units
     {
         // (only when this kernel also combines: a separate combine pass assumes the full grid)
         const long long want = p.pair_cnt ? (U + MIN_UNITS - 1) / MIN_UNITS : p.n_cta;
         cx.n_cta = (int)(want < p.n_cta ? want : p.n_cta);
     }
-    if ((int)blockIdx.x >= cx.n_cta) return;
-    long long lo, hi;
-    if (p.pair_cnt) {
+    if ((int)blockIdx.x >= cx.n_cta) active = false;
+    if (!active) {
+    } else if (p.pair_cnt) {
         // weighted lengths of the scenes (one warp scans them)
         cx.npre = p.P / TILE;
         if (threadIdx.x < 32) {
@@ -1073,39 +1106,10 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, con
         lo = cta_first_unit(blockIdx.x, U, cx.n_cta);
         hi = cta_first_unit(blockIdx.x + 1, U, cx.n_cta);
     }
-    if (lo >= hi) return;
-    if (threadIdx.x == 0) {
-        for (int i = 0; i < MAXST; ++i) {
-            mbar_init(cx.k_full + 8 * i, 1);
-            mbar_init(cx.k_empty + 8 * i, 1);
-            mbar_init(cx.v_full + 8 * i, 1);
-            mbar_init(cx.v_empty + 8 * i, 1);
-        }
-        for (int i = 0; i < 4; ++i) {
-            mbar_init(cx.s_full + 8 * i, 1);
-            mbar_init(cx.s_free + 8 * i, NSOFT);
-        }
-        for (int i = 0; i < 2; ++i) {
-            mbar_init(cx.p_full + 8 * i, NSOFT);
-            mbar_init(cx.pv_done + 8 * i, 1);
-        }
-        mbar_init(cx.q_ready, NSOFT);
-        mbar_init(cx.o_free, NSOFT);
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        fence_async_smem();
-    }
-    if (warp == W_QK) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_holder)), "r"(TMEM_COLS)
-                     : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-    }
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
-    const uint32_t tmem = *reinterpret_cast<volatile uint32_t*>(tmem_holder);
-    cx.tmem = tmem;
+    if (lo >= hi) active = false;
 
-    if (warp == W_KPROD) {
+    if (!active) {
+    } else if (warp == W_KPROD) {
         producer_loop(p, cx, &tm_k, cx.kring, cx.k_full, cx.k_empty, nk, lo, hi, lane);
     } else if (warp == W_VPROD) {
         producer_loop(p, cx, &tm_v, cx.vring, cx.v_full, cx.v_empty, nv, lo, hi, lane);
