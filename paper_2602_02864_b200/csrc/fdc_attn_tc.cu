@@ -811,7 +811,24 @@ __device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& 
             // References are set in the first round of a segment.  Later a score more than 2^16 above its
             // reference only leaves a note (no barrier in the common path): p stays far from overflow, and
             // two rounds later, when all warps are known to see the note, the references are raised.
-            if (t == 0 || (g >= 2 && cx.rflag[(g - 2) & 3] == (int)(g - 2))) {
+            if (t == 0 && __shfl_sync(0xffffffffu, my_tile, k & 31) * TILE + TILE <= p.P) {
+                // First round of a segment inside the prefix: every column takes its score against the
+                // round's first KV row (visible to all) as reference.  That row's own term is then exactly
+                // 1, so no column sum can vanish; higher scores are handled by the lazy raise as usual.
+                if (q4 == 0 && !dead) {                               // the warps that hold TMEM lane 0
+#pragma unroll 1
+                    for (int ch = 0; ch < nch; ++ch) {
+                        uint32_t sv[8];
+                        tmem_ld<8>(s_addr + ch * 8, sv);
+                        tmem_wait_ld();
+                        if (lane == 0) {
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) cx.mneg[col0 + ch * 8 + i] = -(__uint_as_float(sv[i]) * c);
+                        }
+                    }
+                }
+                soft_sync();
+            } else if (t == 0 || (g >= 2 && cx.rflag[(g - 2) & 3] == (int)(g - 2))) {
                 RaiseArgs ra;
                 ra.mneg = cx.mneg;
                 ra.abortp = cx.abortp;
@@ -853,12 +870,21 @@ __device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& 
                     for (int i = 0; i < 8; ++i) {
                         e[i] = fast_exp2(fmaf(__uint_as_float(sv[i]), c, mn[i]));
                         emax = fmaxf(emax, e[i]);
-                        lv[i] = __float_as_uint(__uint_as_float(lv[i]) + e[i]);
+                    }
+                    // P^T goes to the tensor core as bf16; the column sums add up the SAME rounded values, so
+                    // numerator and denominator of the softmax stay consistent (the rounding cancels where a
+                    // few terms dominate)
+                    uint32_t pk[4];
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        pk[j] = pack2(e[2 * j], e[2 * j + 1]);
+                        lv[2 * j] = __float_as_uint(__uint_as_float(lv[2 * j]) + __uint_as_float(pk[j] << 16));
+                        lv[2 * j + 1] = __float_as_uint(__uint_as_float(lv[2 * j + 1]) + __uint_as_float(pk[j] & 0xffff0000u));
                     }
                     tmem_st<8>(l_addr + ch * 8, lv);
                     const int cidx = (col0 >> 3) + ch;                 // 16-byte chunk of the P^T row
                     *reinterpret_cast<uint4*>(prow + (cidx >> 3) * PANEL + (((cidx & 7) ^ (krow & 7)) << 4)) =
-                        make_uint4(pack2(e[0], e[1]), pack2(e[2], e[3]), pack2(e[4], e[5]), pack2(e[6], e[7]));
+                        make_uint4(pk[0], pk[1], pk[2], pk[3]);
                 }
                 tmem_wait_st();
                 if (emax > 65536.f) {                                  // 2^16 above the reference: note it for round g + 2
