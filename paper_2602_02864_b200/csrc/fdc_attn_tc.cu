@@ -58,6 +58,7 @@ constexpr float UNSET = 1.0e30f;             // -reference of a column that has 
 constexpr int W_MASKED = FDC_W_MASKED;       // cost of a tile beyond the prefix (bitmap selects, V clean-up) in prefix tiles
 constexpr int W_PAIR = FDC_W_PAIR;           // cost of finishing a (scene, KV head) pair (drain, partial write, next queries)
 constexpr int MIN_UNITS = 8;                 // tiles per CTA below which fewer CTAs are used (small problems)
+static_assert(MIN_UNITS >= 2 * FDC_W_MASKED, "every part of a pair must contain the start of at least one tile");
 constexpr int MBUF = 512;                    // bitmap words of a scene kept in shared memory (max_active * W)
 
 // ---------------------------------------------------------------- tcgen05 wrappers
@@ -187,7 +188,8 @@ struct Ctx {
     uint64_t* smask;                 // [MBUF] the current segment's scene bitmaps (when mstaged)
     int mstaged;
     int n_cta;                       // CTAs that take part: at most the grid, at least MIN_UNITS tiles each
-    int* prev;                       // [batch + 1] prefix sums of the scenes' weighted lengths (per KV head), or nullptr
+    int* prev;                       // [batch + 1] prefix sums over scenes (per KV head) of parts (tpart > 0) or weighted lengths; or nullptr
+    int tpart;                       // > 0: every CTA owns one part (at most tpart tiles) of one pair
     int npre;                        // tiles wholly inside the prefix
     long long vtot;                  // total weighted length
     volatile int* abortp;
@@ -230,6 +232,13 @@ __device__ __forceinline__ int vt_of(const Ctx& cx, int nt, int j)
     const int np = cx.npre < nt ? cx.npre : nt;
     return j <= np ? j : np + (j - np) * W_MASKED;
 }
+// First tile of a pair of nt tiles whose weighted start is >= r (nt if there is none).
+__device__ __forceinline__ int tile_of_vt(const Ctx& cx, int nt, int r)
+{
+    const int np = cx.npre < nt ? cx.npre : nt;
+    const int j = r <= np ? r : np + (r - np + W_MASKED - 1) / W_MASKED;
+    return j > nt ? nt : j;
+}
 // First unit whose weighted start is >= x.
 __device__ __forceinline__ long long unit_of_virt(const AttnParams& p, const Ctx& cx, long long x)
 {
@@ -245,18 +254,25 @@ __device__ __forceinline__ long long unit_of_virt(const AttnParams& p, const Ctx
     const int V = cx.prev[s + 1] - cx.prev[s], nt = cx.pre[s + 1] - cx.pre[s];
     const long long y = x - (long long)cx.prev[s] * p.hkv;
     const int g = (int)(y / V), r = (int)(y - (long long)g * V);
-    const int np = cx.npre < nt ? cx.npre : nt;
-    int j = r <= np ? r : np + (r - np + W_MASKED - 1) / W_MASKED;
-    if (j > nt) j = nt;
-    return (long long)cx.pre[s] * p.hkv + (long long)g * nt + j;
+    return (long long)cx.pre[s] * p.hkv + (long long)g * nt + tile_of_vt(cx, nt, r);
 }
-// CTA that owns tile j of pair (s, g).
-__device__ __forceinline__ int cta_of_tile(const AttnParams& p, const Ctx& cx, int s, int g, int j)
+// CTAs that hold the first and the last tile of pair (s, g).
+__device__ __forceinline__ void pair_ctas(const AttnParams& p, const Ctx& cx, int s, int g, int& c_first, int& c_last)
 {
     const int nt = cx.pre[s + 1] - cx.pre[s];
-    if (!cx.prev) return unit_cta((long long)cx.pre[s] * p.hkv + (long long)g * nt + j, (long long)cx.pre[p.batch] * p.hkv, cx.n_cta);
-    const long long v = (long long)cx.prev[s] * p.hkv + (long long)g * (cx.prev[s + 1] - cx.prev[s]) + vt_of(cx, nt, j);
-    return (int)((v * cx.n_cta) / cx.vtot);
+    if (cx.tpart) {                                // one part per CTA: the pair's parts are consecutive CTAs
+        const int k = cx.prev[s + 1] - cx.prev[s];
+        c_first = cx.prev[s] * p.hkv + g * k;
+        c_last = c_first + k - 1;
+    } else if (!cx.prev) {
+        const long long u0 = (long long)cx.pre[s] * p.hkv + (long long)g * nt, U = (long long)cx.pre[p.batch] * p.hkv;
+        c_first = unit_cta(u0, U, cx.n_cta);
+        c_last = unit_cta(u0 + nt - 1, U, cx.n_cta);
+    } else {
+        const long long v0 = (long long)cx.prev[s] * p.hkv + (long long)g * (cx.prev[s + 1] - cx.prev[s]);
+        c_first = (int)((v0 * cx.n_cta) / cx.vtot);
+        c_last = (int)(((v0 + vt_of(cx, nt, nt - 1)) * cx.n_cta) / cx.vtot);
+    }
 }
 
 // One TMA producer warp: streams the K (or V) tiles of this CTA's units into its ring, two tiles
@@ -268,6 +284,7 @@ __device__ __forceinline__ void producer_loop(const AttnParams& p, const Ctx& cx
     uint32_t g = 0;
     long long u = lo;
     int ok = 1;
+    const uint64_t pol = l2_evict_first_policy();     // every KV row is read once per call
     while (u < hi && ok) {
         const Segment sg = decode_segment(u, hi, cx.pre, p.hkv, s);
         for (int jb = sg.j0; jb < sg.j1 && ok; jb += 32) {
@@ -286,8 +303,8 @@ __device__ __forceinline__ void producer_loop(const AttnParams& p, const Ctx& cx
                         mbar_expect_tx(full + 8 * st, nt * (STAGE / 2));
 #pragma unroll
                         for (int h = 0; h < D / 64; ++h) {
-                            tma_load_4d(dst + h * PANEL, tm, full + 8 * st, h * 64, t0 * TILE, sg.g, sg.s);
-                            if (nt == 2) tma_load_4d(dst + h * PANEL + TILE * 128, tm, full + 8 * st, h * 64, t1 * TILE, sg.g, sg.s);
+                            tma_load_4d_hint(dst + h * PANEL, tm, full + 8 * st, h * 64, t0 * TILE, sg.g, sg.s, pol);
+                            if (nt == 2) tma_load_4d_hint(dst + h * PANEL + TILE * 128, tm, full + 8 * st, h * 64, t1 * TILE, sg.g, sg.s, pol);
                         }
                     }
                 }
@@ -983,7 +1000,8 @@ __device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& 
             __threadfence();
             soft_sync();
             if (tid == 0) {
-                const int c_first = cta_of_tile(p, cx, sg.s, sg.g, 0), c_last = cta_of_tile(p, cx, sg.s, sg.g, sg.nt - 1);
+                int c_first, c_last;
+                pair_ctas(p, cx, sg.s, sg.g, c_first, c_last);
                 const int expected = c_last - c_first + 1;               // every CTA in between owns tiles of the pair
                 const int old = dead ? -1 : atomicAdd(&p.pair_cnt[pair], 1);
                 cx.flags[1] = old == expected - 1;
@@ -1092,25 +1110,67 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, con
     const long long total = scan_ntiles(p.ntiles, p.batch, cx.pre);
     const long long U = total * p.hkv;
     if (U == 0) active = false;
-    // small problems use fewer CTAs (fewer partials to merge); every participating CTA owns units
-    {
-        // (only when this kernel also combines: a separate combine pass assumes the full grid)
-        const long long want = p.pair_cnt ? (U + MIN_UNITS - 1) / MIN_UNITS : p.n_cta;
-        cx.n_cta = (int)(want < p.n_cta ? want : p.n_cta);
-    }
-    if ((int)blockIdx.x >= cx.n_cta) active = false;
+    cx.tpart = 0;
+    cx.n_cta = p.n_cta;
     if (!active) {
     } else if (p.pair_cnt) {
-        // weighted lengths of the scenes (one warp scans them)
+        // This kernel also merges the partial results of a pair.  Ending one pair and starting the
+        // next inside a CTA costs as much as streaming a dozen tiles (drain, partial write, merge,
+        // new queries), so while there are no more pairs than CTAs every CTA gets ONE part of ONE
+        // pair: pairs are cut into the fewest equal parts of at most tpart (weighted) tiles, tpart the smallest
+        // size (at least MIN_UNITS) for which the parts do not outnumber the CTAs.  With more pairs
+        // than CTAs, CTAs get equal shares of a weighted length (see above).
         cx.npre = p.P / TILE;
+        __shared__ int split_tpart, split_max, split_pairs;
+        if (threadIdx.x == 0) {
+            split_tpart = 0x7fffffff;
+            split_max = 0;
+            split_pairs = 0;
+        }
+        __syncthreads();
+        {
+            int nsc = 0, mx = 0;
+            for (int i = threadIdx.x; i < p.batch; i += THREADS) {
+                const int nt = cx.pre[i + 1] - cx.pre[i];
+                nsc += nt > 0;
+                mx = nt > mx ? nt : mx;
+            }
+            if (nsc) {
+                atomicAdd(&split_pairs, nsc);
+                atomicMax(&split_max, mx);
+            }
+        }
+        __syncthreads();
+        const bool one_part = (long long)split_pairs * p.hkv <= p.n_cta;
+        if (one_part) {
+            // every thread tries sizes of its own; the smallest that fits wins
+            const uint32_t vmax = (uint32_t)vt_of(cx, split_max, split_max);
+            const uint32_t tl = vmax < (uint32_t)MIN_UNITS ? vmax : (uint32_t)MIN_UNITS;
+            const uint32_t budget = (uint32_t)(p.n_cta / p.hkv);          // parts per KV head
+            for (uint32_t T = tl + threadIdx.x; T <= vmax && T < (uint32_t)split_tpart; T += THREADS) {
+                uint32_t cnt = 0;
+                for (int i = 0; i < p.batch; ++i) {
+                    const int nt = cx.pre[i + 1] - cx.pre[i];
+                    cnt += ((uint32_t)vt_of(cx, nt, nt) + T - 1) / T;
+                }
+                if (cnt <= budget) {
+                    atomicMin(&split_tpart, (int)T);
+                    break;
+                }
+            }
+        } else if (threadIdx.x == 0) {
+            split_tpart = 0;
+        }
+        __syncthreads();
         if (threadIdx.x < 32) {
+            const uint32_t T = (uint32_t)split_tpart;
             int carry = 0;
             for (int b0 = 0; b0 < p.batch; b0 += 32) {
                 const int i = b0 + threadIdx.x;
                 int x = 0;
                 if (i < p.batch) {
                     const int nt = cx.pre[i + 1] - cx.pre[i];
-                    x = nt > 0 ? vt_of(cx, nt, nt) + W_PAIR : 0;
+                    x = T ? (int)(((uint32_t)vt_of(cx, nt, nt) + T - 1) / T) : (nt > 0 ? vt_of(cx, nt, nt) + W_PAIR : 0);
                 }
                 int inc = x;
 #pragma unroll
@@ -1124,15 +1184,39 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, con
             if (threadIdx.x == 0) cx.prev[p.batch] = carry;
         }
         __syncthreads();
-        cx.vtot = (long long)cx.prev[p.batch] * p.hkv;
-        lo = unit_of_virt(p, cx, cta_first_unit(blockIdx.x, cx.vtot, cx.n_cta));
-        hi = unit_of_virt(p, cx, cta_first_unit(blockIdx.x + 1, cx.vtot, cx.n_cta));
+        cx.tpart = split_tpart;
+        if (cx.tpart) {
+            const int c = blockIdx.x;
+            cx.n_cta = cx.prev[p.batch] * p.hkv;
+            if (c < cx.n_cta) {
+                int sl = 0, sh = p.batch;              // largest s with prev[s] * hkv <= c
+                while (sh - sl > 1) {
+                    const int mid = (sl + sh) >> 1;
+                    if (cx.prev[mid] * p.hkv <= c) sl = mid;
+                    else sh = mid;
+                }
+                while (cx.prev[sl + 1] == cx.prev[sl]) ++sl;          // scenes without tiles have no parts
+                const int k = cx.prev[sl + 1] - cx.prev[sl], nt = cx.pre[sl + 1] - cx.pre[sl];
+                const uint32_t idx = (uint32_t)(c - cx.prev[sl] * p.hkv), g = idx / (uint32_t)k, i = idx - g * (uint32_t)k;
+                const uint32_t V = (uint32_t)vt_of(cx, nt, nt);       // part i: tiles whose weighted start lies in [i V / k, (i + 1) V / k)
+                const int j0 = tile_of_vt(cx, nt, (int)((i * V + k - 1) / (uint32_t)k));
+                const int j1 = tile_of_vt(cx, nt, (int)(((i + 1) * V + k - 1) / (uint32_t)k));
+                lo = (long long)cx.pre[sl] * p.hkv + (long long)g * nt + j0;
+                hi = lo + (j1 - j0);
+            }
+        } else {
+            const long long want = (U + MIN_UNITS - 1) / MIN_UNITS;      // small problems use fewer CTAs
+            if (want < cx.n_cta) cx.n_cta = (int)want;
+            cx.vtot = (long long)cx.prev[p.batch] * p.hkv;
+            lo = unit_of_virt(p, cx, cta_first_unit(blockIdx.x, cx.vtot, cx.n_cta));
+            hi = unit_of_virt(p, cx, cta_first_unit(blockIdx.x + 1, cx.vtot, cx.n_cta));
+        }
     } else {
         cx.prev = nullptr;
         lo = cta_first_unit(blockIdx.x, U, cx.n_cta);
         hi = cta_first_unit(blockIdx.x + 1, U, cx.n_cta);
     }
-    if (lo >= hi) active = false;
+    if (lo >= hi || (int)blockIdx.x >= cx.n_cta) active = false;
 
     if (!active) {
     } else if (warp == W_KPROD) {
