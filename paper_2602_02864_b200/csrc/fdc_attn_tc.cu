@@ -39,7 +39,7 @@ constexpr int TILE = FDC_TILE_ROWS;          // rows per entry of the visited-ti
 constexpr int RROWS = 2 * TILE;              // KV rows per round = M of S^T = K of O^T
 constexpr int NSOFT = 16;                    // softmax warps: 4 row quadrants x 4 column parts
 constexpr int NPART = NSOFT / 4;             // column parts
-constexpr int W_KPROD = NSOFT, W_QK = NSOFT + 1, W_VPROD = NSOFT + 2, W_PV = NSOFT + 3;
+constexpr int W_PROD = NSOFT, W_QK = NSOFT + 1, W_CLEAN = NSOFT + 2, W_PV = NSOFT + 3;
 constexpr int THREADS = (NSOFT + 4) * 32;
 constexpr uint32_t TMEM_COLS = 512;          // S^T 0 [0,128) | S^T 1 [128,256) | O^T [256,384) | sums [384,512)
 constexpr uint32_t TM_O = 256;
@@ -57,6 +57,7 @@ constexpr float UNSET = 1.0e30f;             // -reference of a column that has 
 #endif
 constexpr int W_MASKED = FDC_W_MASKED;       // cost of a tile beyond the prefix (bitmap selects, V clean-up) in prefix tiles
 constexpr int W_PAIR = FDC_W_PAIR;           // cost of finishing a (scene, KV head) pair (drain, partial write, next queries)
+constexpr int UW = 64;                       // words of a scene's union bitmap kept in shared memory (when W <= UW)
 constexpr int MIN_UNITS = 8;                 // tiles per CTA below which fewer CTAs are used (small problems)
 static_assert(MIN_UNITS >= 2 * FDC_W_MASKED, "every part of a pair must contain the start of at least one tile");
 constexpr int MBUF = 512;                    // bitmap words of a scene kept in shared memory (max_active * W)
@@ -177,7 +178,7 @@ __device__ __forceinline__ float ord_to(int i) { return __int_as_float(i ^ ((i >
 
 // Everything a role needs to find its barriers and buffers.
 struct Ctx {
-    uint32_t k_full, k_empty, v_full, v_empty, s_full, s_free, p_full, pv_done, q_ready, o_free;
+    uint32_t k_full, k_empty, v_full, v_empty, v_clean, s_full, s_free, p_full, pv_done, q_ready, o_free;
     int ns, s_stride;                // S^T buffers in TMEM (4 of 64 columns up to 64 query rows, else 2 of 128) and their distance
     uint32_t tmem;
     unsigned char *kring, *vring, *qs, *ps;
@@ -185,7 +186,8 @@ struct Ctx {
     int *cmax, *flags;               // [128] column maxima (ordered ints), [4] flags of the raise path and the merge
     int* rflag;                      // [4] rflag[g & 3] == g: round g met a score far above its reference
     int *pre, *nact;                 // [batch + 1] tile prefix sums, [batch] active branches per scene
-    uint64_t* smask;                 // [MBUF] the current segment's scene bitmaps (when mstaged)
+    uint64_t* smask;                 // [2][MBUF] the current segment's scene bitmaps (when mstaged)
+    uint64_t* sunion;                // [2][UW] their OR over the scene's active branches (when mstaged and W <= UW)
     int mstaged;
     int n_cta;                       // CTAs that take part: at most the grid, at least MIN_UNITS tiles each
     int* prev;                       // [batch + 1] prefix sums over scenes (per KV head) of parts (tpart > 0) or weighted lengths; or nullptr
@@ -275,50 +277,122 @@ __device__ __forceinline__ void pair_ctas(const AttnParams& p, const Ctx& cx, in
     }
 }
 
-// One TMA producer warp: streams the K (or V) tiles of this CTA's units into its ring, two tiles
-// per stage (rows 0-63 and 64-127 of both 64-column panels).
-__device__ __forceinline__ void producer_loop(const AttnParams& p, const Ctx& cx, const CUtensorMap* tm, unsigned char* ring,
-                                              uint32_t full, uint32_t empty, int nst, long long lo, long long hi, int lane)
+// Position of one ring's producer in the CTA's unit sequence.
+struct Cursor {
+    long long u;                 // first unit of the current segment
+    Segment sg;
+    int s, jb, jn, k, my_tile;   // scene hint; batch of up to 32 tile ids (one per lane) and the position inside it
+    uint32_t g;                  // round
+    int st;                      // ring stage of round g
+    uint32_t ph;                 // ring phase of round g
+    int live;
+};
+__device__ __forceinline__ void cursor_batch(Cursor& c, const AttnParams& p, int lane)
 {
-    int s = 0;
-    uint32_t g = 0;
-    long long u = lo;
-    int ok = 1;
-    const uint64_t pol = l2_evict_first_policy();     // every KV row is read once per call
-    while (u < hi && ok) {
-        const Segment sg = decode_segment(u, hi, cx.pre, p.hkv, s);
-        for (int jb = sg.j0; jb < sg.j1 && ok; jb += 32) {
-            const int jn = sg.j1 - jb < 32 ? sg.j1 - jb : 32;
-            const int my_tile = lane < jn ? p.tiles[(size_t)sg.s * p.ntile_max + jb + lane] : 0;
-            for (int k = 0; k < jn && ok; k += 2, ++g) {
-                const int nt = jn - k < 2 ? 1 : 2;
-                const int t0 = __shfl_sync(0xffffffffu, my_tile, k);
-                const int t1 = __shfl_sync(0xffffffffu, my_tile, (k + 1) & 31);
-                if (lane == 0) {
-                    const int st = g % nst;
-                    if (!mbar_wait(empty + 8 * st, ((g / nst) & 1) ^ 1, cx.abortp, p.status)) {
-                        ok = 0;
-                    } else {
-                        const uint32_t dst = smem_u32(ring + (size_t)st * STAGE);
-                        mbar_expect_tx(full + 8 * st, nt * (STAGE / 2));
+    c.jn = c.sg.j1 - c.jb < 32 ? c.sg.j1 - c.jb : 32;
+    c.my_tile = lane < c.jn ? p.tiles[(size_t)c.sg.s * p.ntile_max + c.jb + lane] : 0;
+    c.k = 0;
+}
+__device__ __forceinline__ void cursor_open(Cursor& c, const AttnParams& p, const Ctx& cx, long long hi, int lane)
+{
+    c.live = c.u < hi;
+    if (!c.live) return;
+    c.sg = decode_segment(c.u, hi, cx.pre, p.hkv, c.s);
+    c.jb = c.sg.j0;
+    cursor_batch(c, p, lane);
+}
+__device__ __forceinline__ void cursor_next(Cursor& c, const AttnParams& p, const Ctx& cx, long long hi, int nst, int lane)
+{
+    c.k += 2;
+    ++c.g;
+    if (++c.st == nst) {
+        c.st = 0;
+        c.ph ^= 1;
+    }
+    if (c.k < c.jn) return;
+    c.jb += 32;
+    if (c.jb < c.sg.j1) {
+        cursor_batch(c, p, lane);
+    } else {
+        c.u = c.sg.next_u;
+        cursor_open(c, p, cx, hi, lane);
+    }
+}
+// The round at the cursor: two tiles (rows 0-63 and 64-127 of both 64-column panels) into one stage.
+__device__ __forceinline__ void cursor_issue(const Cursor& c, const CUtensorMap* tm, unsigned char* ring, uint32_t full, uint64_t pol, int lane)
+{
+    const int nt = c.jn - c.k < 2 ? 1 : 2;
+    const int t0 = __shfl_sync(0xffffffffu, c.my_tile, c.k);
+    const int t1 = __shfl_sync(0xffffffffu, c.my_tile, (c.k + 1) & 31);
+    if (lane == 0) {
+        const uint32_t dst = smem_u32(ring + (size_t)c.st * STAGE);
+        mbar_expect_tx(full + 8 * c.st, nt * (STAGE / 2));
 #pragma unroll
-                        for (int h = 0; h < D / 64; ++h) {
-                            tma_load_4d_hint(dst + h * PANEL, tm, full + 8 * st, h * 64, t0 * TILE, sg.g, sg.s, pol);
-                            if (nt == 2) tma_load_4d_hint(dst + h * PANEL + TILE * 128, tm, full + 8 * st, h * 64, t1 * TILE, sg.g, sg.s, pol);
-                        }
-                    }
+        for (int h = 0; h < D / 64; ++h) {
+            tma_load_4d_hint(dst + h * PANEL, tm, full + 8 * c.st, h * 64, t0 * TILE, c.sg.g, c.sg.s, pol);
+            if (nt == 2) tma_load_4d_hint(dst + h * PANEL + TILE * 128, tm, full + 8 * c.st, h * 64, t1 * TILE, c.sg.g, c.sg.s, pol);
+        }
+    }
+}
+
+// One TMA producer warp for both rings: whichever of the next K stage and the next V stage is
+// free gets its round's tiles; the warp never blocks on one ring while the other could be fed.
+__device__ __forceinline__ void producer_loop(const AttnParams& p, const Ctx& cx, const CUtensorMap* tm_k, const CUtensorMap* tm_v,
+                                              long long lo, long long hi, int lane)
+{
+    const uint64_t pol = l2_evict_first_policy();     // every KV row is read once per call
+    Cursor ck, cv;
+    ck.u = lo;
+    ck.s = 0;
+    ck.g = 0;
+    ck.st = 0;
+    ck.ph = 0;
+    cursor_open(ck, p, cx, hi, lane);
+    cv = ck;
+    int ok = 1;
+    uint32_t idle = 0;
+    while ((ck.live || cv.live) && ok) {
+        int rk = 0, rv = 0;
+        if (lane == 0) {
+            rk = ck.live && mbar_try(cx.k_empty + 8 * ck.st, ck.ph ^ 1);
+            rv = cv.live && mbar_try(cx.v_empty + 8 * cv.st, cv.ph ^ 1);
+        }
+        rk = __shfl_sync(0xffffffffu, rk, 0);
+        rv = __shfl_sync(0xffffffffu, rv, 0);
+        if (rk) {
+            cursor_issue(ck, tm_k, cx.kring, cx.k_full, pol, lane);
+            cursor_next(ck, p, cx, hi, cx.nk, lane);
+        }
+        if (rv) {
+            cursor_issue(cv, tm_v, cx.vring, cx.v_full, pol, lane);
+            cursor_next(cv, p, cx, hi, cx.nv, lane);
+        }
+        if (rk | rv) {
+            idle = 0;
+        } else if (((++idle) & 63u) == 0u) {
+            // bounded: no stage became free for a long time, or another role gave up
+            if (idle >= SPIN_LIMIT) {
+                if (lane == 0) {
+                    *cx.abortp = 1;
+                    atomicOr(p.status, FDC_DEV_TIMEOUT);
                 }
-                ok = __shfl_sync(0xffffffffu, ok, 0);
+                ok = 0;
+            } else if (*cx.abortp) {
+                ok = 0;
+            } else {
+                __nanosleep(32);
             }
         }
-        u = sg.next_u;
     }
     if (!ok && lane == 0) {
         // give the copies already in flight a bounded chance to land before the CTA ends
-        const uint32_t first = g > (uint32_t)nst ? g - nst : 0;
-        for (uint32_t k = first; k < g; ++k) {
-            const uint32_t bar = full + 8 * (k % nst), ph = (k / nst) & 1;
-            for (uint32_t i = 0; i < (1u << 16) && !mbar_try(bar, ph); ++i) __nanosleep(64);
+        for (int r = 0; r < 2; ++r) {
+            const uint32_t g = r ? cv.g : ck.g, nst = r ? cx.nv : cx.nk, full = r ? cx.v_full : cx.k_full;
+            const uint32_t first = g > nst ? g - nst : 0;
+            for (uint32_t k = first; k < g; ++k) {
+                const uint32_t bar = full + 8 * (k % nst), ph = (k / nst) & 1;
+                for (uint32_t i = 0; i < (1u << 16) && !mbar_try(bar, ph); ++i) __nanosleep(64);
+            }
         }
     }
 }
@@ -377,32 +451,40 @@ __device__ __forceinline__ void qk_loop(const AttnParams& p, const Ctx& cx, long
 }
 
 // V rows of a stage that are invisible to every branch of the scene are cleared (whole warp; kept
-// out of line: only rounds beyond the prefix come here).  tile0 / tile1 are the round's tiles.
-__device__ __noinline__ void clear_unseen_rows(unsigned char* vs, const uint64_t* mask0, int W, int P, int A, int tile0, int tile1, int nt)
+// out of line: only rounds beyond the prefix come here).  tile0 / tile1 are the round's tiles, vs
+// the stage's shared-memory address.  `un` is the OR of the scene's bitmaps when the softmax warps
+// have prepared it (the usual case), else nullptr and the bitmaps themselves are combined here.
+__device__ __noinline__ void clear_unseen_rows(uint32_t vs, const uint64_t* un, const uint64_t* mask0, int W, int P, int A, int tile0, int tile1, int nt)
 {
     const int lane = threadIdx.x & 31;
     bool touched = false;
     for (int i = 0; i < nt; ++i) {
         const int tile = i ? tile1 : tile0;
         if (tile * TILE + TILE <= P) continue;                 // all rows visible to everybody
-        uint64_t um = 0ull;
-        for (int b = lane; b < A; b += 32) um |= tile_rowmask(mask0 + (size_t)b * W, W, P, tile);
-        const uint32_t ul = __reduce_or_sync(0xffffffffu, (uint32_t)um);
-        const uint32_t uh = __reduce_or_sync(0xffffffffu, (uint32_t)(um >> 32));
-        const uint64_t z = ~(((uint64_t)uh << 32) | ul);
+        uint64_t seen;
+        if (un) {
+            seen = tile_rowmask(un, W, P, tile);
+        } else {
+            uint64_t um = 0ull;
+            for (int b = lane; b < A; b += 32) um |= tile_rowmask(mask0 + (size_t)b * W, W, P, tile);
+            const uint32_t ul = __reduce_or_sync(0xffffffffu, (uint32_t)um);
+            const uint32_t uh = __reduce_or_sync(0xffffffffu, (uint32_t)(um >> 32));
+            seen = ((uint64_t)uh << 32) | ul;
+        }
+        const uint64_t z = ~seen;
         if (z) {
             // lane l clears rows l and l + 32 of the tile if nobody sees them (2 panels x 8 chunks of 16 bytes)
 #pragma unroll
             for (int hr = 0; hr < 2; ++hr) {
                 const int r = lane + 32 * hr;
                 if ((z >> r) & 1) {
-                    unsigned char* row = vs + (i * TILE + r) * 128;
+                    const uint32_t row = vs + (i * TILE + r) * 128;
 #pragma unroll
                     for (int ch = 0; ch < 8; ++ch) {
                         // rotate the chunk order by the row so that the lanes of a warp hit different banks
-                        const int cc = ((ch + r) & 7) << 4;
-                        *reinterpret_cast<uint4*>(row + cc) = make_uint4(0u, 0u, 0u, 0u);
-                        *reinterpret_cast<uint4*>(row + PANEL + cc) = make_uint4(0u, 0u, 0u, 0u);
+                        const uint32_t cc = ((ch + r) & 7) << 4;
+                        asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(row + cc), "r"(0u) : "memory");
+                        asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(row + PANEL + cc), "r"(0u) : "memory");
                     }
                 }
             }
@@ -413,10 +495,56 @@ __device__ __noinline__ void clear_unseen_rows(unsigned char* vs, const uint64_t
     __syncwarp();
 }
 
-// Warp 11: O^T += V^T(stage) P^T[g & 1] for every round g (one elected thread issues).  Before
-// that the whole warp clears the V rows of the stage that are invisible to every branch of the
-// scene: their P^T row is exactly 0, but the rows can hold anything (NaN, Inf) and 0 * NaN must
-// not reach the accumulator.  Stages wholly inside the prefix need no such pass.
+// One warp: the V rows of a stage that are invisible to every branch of the scene are cleared
+// before the stage is multiplied.  Their P^T row is exactly 0, but the rows can hold anything
+// (NaN, Inf: slots that were never written) and 0 * NaN must not reach the accumulator.  Stages
+// wholly inside the prefix are passed on as they are.  A warp of its own, so that the clean-up
+// runs ahead (as far as the V ring is deep) instead of delaying the multiplications.
+__device__ __forceinline__ void clean_loop(const AttnParams& p, const Ctx& cx, long long lo, long long hi, int lane)
+{
+    int s = 0;
+    uint32_t seg = 0;
+    int st = 0;
+    uint32_t vph = 0;
+    long long u = lo;
+    int ok = 1;
+    while (u < hi && ok) {
+        const Segment sg = decode_segment(u, hi, cx.pre, p.hkv, s);
+        const int A = cx.nact[sg.s];
+        bool have_masks = !cx.mstaged;                 // staged bitmaps are published with the queries (q_ready)
+        for (int jb = sg.j0; jb < sg.j1 && ok; jb += 32) {
+            const int jn = sg.j1 - jb < 32 ? sg.j1 - jb : 32;
+            const int my_tile = lane < jn ? p.tiles[(size_t)sg.s * p.ntile_max + jb + lane] : 0;
+            for (int k = 0; k < jn && ok; k += 2) {
+                const int nt = jn - k < 2 ? 1 : 2;
+                // tile ids ascend: the round reaches beyond the prefix iff its last tile does
+                const int t_last = __shfl_sync(0xffffffffu, my_tile, (k + nt - 1) & 31);
+                const bool masked = t_last * TILE + TILE > p.P;
+                int okw = 1;
+                if (lane == 0) {
+                    okw = mbar_wait(cx.v_full + 8 * st, vph, cx.abortp, p.status);
+                    if (okw && masked && !have_masks) okw = mbar_wait(cx.q_ready, seg & 1, cx.abortp, p.status);
+                }
+                ok = __shfl_sync(0xffffffffu, okw, 0);
+                if (ok && masked) {
+                    have_masks = true;
+                    clear_unseen_rows(smem_u32(cx.vring) + st * STAGE, (cx.mstaged && p.W <= UW) ? cx.sunion + (seg & 1) * UW : nullptr,
+                                      mask_row(p, cx, seg, sg.s, 0), p.W, p.P, A, __shfl_sync(0xffffffffu, my_tile, k & 31), t_last, nt);
+                }
+                if (ok && lane == 0) mbar_arrive(cx.v_clean + 8 * st);
+                if (++st == cx.nv) {
+                    st = 0;
+                    vph ^= 1;
+                }
+            }
+        }
+        ++seg;
+        u = sg.next_u;
+    }
+}
+
+// One elected thread: O^T += V^T(stage) P^T[g & 1] for every round g, once the stage has been
+// passed on by the cleaning warp and the softmax warps have delivered P^T.
 __device__ __forceinline__ void pv_loop(const AttnParams& p, const Ctx& cx, long long lo, long long hi, int lane)
 {
     const uint64_t v_desc0 = smem_desc(smem_u32(cx.vring), PANEL, 1024);
@@ -431,56 +559,40 @@ __device__ __forceinline__ void pv_loop(const AttnParams& p, const Ctx& cx, long
     int ok = 1;
     while (u < hi && ok) {
         const Segment sg = decode_segment(u, hi, cx.pre, p.hkv, s);
-        const int A = cx.nact[sg.s];
-        const int M = A * p.group;
-        const int NP = M <= 32 ? 32 : (M <= 64 ? 64 : 128);
-        const uint32_t idesc_pv = instr_desc(D, NP, 1);
-        if (cx.mstaged) {                            // the softmax warps publish the scene's bitmaps with the queries
-            int okw = 1;
-            if (lane == 0) okw = mbar_wait(cx.q_ready, seg & 1, cx.abortp, p.status);
-            ok = __shfl_sync(0xffffffffu, okw, 0);
-        }
-        int t = 0;
-        for (int jb = sg.j0; jb < sg.j1 && ok; jb += 32) {
-            const int jn = sg.j1 - jb < 32 ? sg.j1 - jb : 32;
-            const int my_tile = lane < jn ? p.tiles[(size_t)sg.s * p.ntile_max + jb + lane] : 0;
-            for (int k = 0; k < jn && ok; k += 2, ++g, ++t) {
-                const int nt = jn - k < 2 ? 1 : 2;
-                // tile ids ascend: the round reaches beyond the prefix iff its last tile does
-                const int t_last = __shfl_sync(0xffffffffu, my_tile, (k + nt - 1) & 31);
-                int okw = 1;
-                if (lane == 0) okw = mbar_wait(cx.v_full + 8 * st, vph, cx.abortp, p.status);
-                if (t_last * TILE + TILE > p.P) {
-                    okw = __shfl_sync(0xffffffffu, okw, 0);
-                    if (okw)
-                        clear_unseen_rows(cx.vring + (size_t)st * STAGE, mask_row(p, cx, seg, sg.s, 0), p.W, p.P, A,
-                                          __shfl_sync(0xffffffffu, my_tile, k & 31), t_last, nt);
-                }
-                if (lane == 0 && okw) {
-                    bool good = mbar_wait(cx.p_full + 8 * (g & 1), (g >> 1) & 1, cx.abortp, p.status);
-                    if (good && t == 0 && seg > 0) good = mbar_wait(cx.o_free, (seg - 1) & 1, cx.abortp, p.status);
-                    if (good) {
-                        tc_fence_after();
-                        const uint32_t vd = v_lo0 + (uint32_t)((st * STAGE) >> 4);
-                        const uint32_t pd = p_lo0 + (uint32_t)((((g & 1) & (cx.npb - 1)) * cx.p_buf) >> 4);
+        if (lane == 0) {
+            const int M = cx.nact[sg.s] * p.group;
+            const int NP = M <= 32 ? 32 : (M <= 64 ? 64 : 128);
+            const uint32_t idesc_pv = instr_desc(D, NP, 1);
+            const int ntile = sg.j1 - sg.j0;
+            bool good = true;
+            for (int t = 0; 2 * t < ntile && good; ++t, ++g) {
+                const int nt = ntile - 2 * t < 2 ? 1 : 2;
+                good = mbar_wait(cx.v_clean + 8 * st, vph, cx.abortp, p.status);
+                if (good) good = mbar_wait(cx.p_full + 8 * (g & 1), (g >> 1) & 1, cx.abortp, p.status);
+                if (good && t == 0 && seg > 0) good = mbar_wait(cx.o_free, (seg - 1) & 1, cx.abortp, p.status);
+                if (!good) break;
+                tc_fence_after();
+                const uint32_t vd = v_lo0 + (uint32_t)((st * STAGE) >> 4);
+                const uint32_t pd = p_lo0 + (uint32_t)((((g & 1) & (cx.npb - 1)) * cx.p_buf) >> 4);
 #pragma unroll
-                        for (int kk = 0; kk < 4; ++kk) umma2(tm_o, vd + kk * 128, v_hi, pd + kk * 128, p_hi, idesc_pv, (t > 0 || kk > 0) ? 1u : 0u);
-                        if (nt == 2) {                                       // a one-tile round has 64 KV rows
+                for (int kk = 0; kk < 4; ++kk) umma2(tm_o, vd + kk * 128, v_hi, pd + kk * 128, p_hi, idesc_pv, (t > 0 || kk > 0) ? 1u : 0u);
+                if (nt == 2) {                                       // a one-tile round has 64 KV rows
 #pragma unroll
-                            for (int kk = 4; kk < 8; ++kk) umma2(tm_o, vd + kk * 128, v_hi, pd + kk * 128, p_hi, idesc_pv, 1u);
-                        }
-                        umma_commit(cx.v_empty + 8 * st);
-                        umma_commit(cx.pv_done + 8 * (g & 1));
-                    }
-                    okw = good;
+                    for (int kk = 4; kk < 8; ++kk) umma2(tm_o, vd + kk * 128, v_hi, pd + kk * 128, p_hi, idesc_pv, 1u);
                 }
-                ok = __shfl_sync(0xffffffffu, okw, 0);
+                umma_commit(cx.v_empty + 8 * st);
+                umma_commit(cx.pv_done + 8 * (g & 1));
                 if (++st == cx.nv) {
                     st = 0;
                     vph ^= 1;
                 }
             }
+            ok = good;
         }
+        ok = __shfl_sync(0xffffffffu, ok, 0);
+        g = __shfl_sync(0xffffffffu, g, 0);
+        st = __shfl_sync(0xffffffffu, st, 0);
+        vph = __shfl_sync(0xffffffffu, vph, 0);
         ++seg;
         u = sg.next_u;
     }
@@ -780,6 +892,16 @@ __device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& 
                 if (idx < nw) cx.smask[(seg & 1) * MBUF + idx] = mv[i];
             }
         }
+        if (cx.mstaged && p.W <= UW) {
+            // OR of the scene's bitmaps: the rows no branch may see, for the warp that cleans V
+            soft_sync();                              // everybody's share of the bitmaps is in place
+            if (tid < p.W) {
+                const uint64_t* mb = cx.smask + (seg & 1) * MBUF + tid;
+                uint64_t un = 0ull;
+                for (int b = 0; b < A; ++b) un |= mb[(size_t)b * p.W];
+                cx.sunion[(seg & 1) * UW + tid] = un;
+            }
+        }
         if (tid < np) cx.mneg[tid] = UNSET;
         {
             uint32_t z[8];
@@ -1042,7 +1164,8 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, con
     cx.k_empty = cx.k_full + 8 * MAXST;
     cx.v_full = cx.k_empty + 8 * MAXST;
     cx.v_empty = cx.v_full + 8 * MAXST;
-    cx.s_full = cx.v_empty + 8 * MAXST;
+    cx.v_clean = cx.v_empty + 8 * MAXST;
+    cx.s_full = cx.v_clean + 8 * MAXST;
     cx.s_free = cx.s_full + 8 * 4;
     cx.p_full = cx.s_free + 8 * 4;
     cx.ns = np_max <= 64 ? 4 : 2;
@@ -1050,7 +1173,7 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, con
     cx.pv_done = cx.p_full + 16;
     cx.q_ready = cx.pv_done + 16;
     cx.o_free = cx.q_ready + 8;
-    uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bars + 4 * MAXST + 14);
+    uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bars + 5 * MAXST + 14);
     cx.mneg = reinterpret_cast<float*>(tmem_holder + 4);
     cx.alpha = cx.mneg + 128;
     cx.lred = cx.alpha + 128;
@@ -1061,6 +1184,7 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, con
     cx.nact = cx.pre + p.batch + 1;
     cx.prev = cx.nact + p.batch;
     cx.smask = reinterpret_cast<uint64_t*>(((uintptr_t)(cx.prev + p.batch + 1) + 7) & ~(uintptr_t)7);
+    cx.sunion = cx.smask + 2 * MBUF;
     cx.mstaged = p.max_active * p.W <= MBUF;
     __shared__ int abort_flag;
     cx.abortp = &abort_flag;
@@ -1075,6 +1199,7 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, con
             mbar_init(cx.k_empty + 8 * i, 1);
             mbar_init(cx.v_full + 8 * i, 1);
             mbar_init(cx.v_empty + 8 * i, 1);
+            mbar_init(cx.v_clean + 8 * i, 1);
         }
         for (int i = 0; i < 4; ++i) {
             mbar_init(cx.s_full + 8 * i, 1);
@@ -1219,10 +1344,10 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, con
     if (lo >= hi || (int)blockIdx.x >= cx.n_cta) active = false;
 
     if (!active) {
-    } else if (warp == W_KPROD) {
-        producer_loop(p, cx, &tm_k, cx.kring, cx.k_full, cx.k_empty, nk, lo, hi, lane);
-    } else if (warp == W_VPROD) {
-        producer_loop(p, cx, &tm_v, cx.vring, cx.v_full, cx.v_empty, nv, lo, hi, lane);
+    } else if (warp == W_PROD) {
+        producer_loop(p, cx, &tm_k, &tm_v, lo, hi, lane);
+    } else if (warp == W_CLEAN) {
+        clean_loop(p, cx, lo, hi, lane);
     } else if (warp == W_PV) {
         pv_loop(p, cx, lo, hi, lane);
     } else if (warp == W_QK) {
@@ -1262,8 +1387,8 @@ int launch_attn_tc(const AttnParams& p, int head_dim, cudaStream_t st)
     const int np_max = p.mmax <= 32 ? 32 : (p.mmax <= 64 ? 64 : 128);
     const int p_buf = ((np_max + 63) / 64) * PANEL;
     const int npb = np_max > 64 ? 1 : 2;          // 128 query rows: one P^T buffer, so that four stages still fit
-    const size_t fixed = 1024 + (size_t)npb * p_buf + (size_t)(D / 64) * np_max * 128 + 8 * (4 * MAXST + 14) + 16 +
-                         4 * (128 + 128 + 512 + 128 + 8) + sizeof(int) * (3 * p.batch + 2) + 8 * (2 * MBUF + 2) + 64;
+    const size_t fixed = 1024 + (size_t)npb * p_buf + (size_t)(D / 64) * np_max * 128 + 8 * (5 * MAXST + 14) + 16 +
+                         4 * (128 + 128 + 512 + 128 + 8) + sizeof(int) * (3 * p.batch + 2) + 8 * (2 * MBUF + 2 * UW + 2) + 64;
     int stages = (int)((227 * 1024 - 256 - fixed) / STAGE);
     if (stages > 2 * MAXST) stages = 2 * MAXST;
     if (stages < 4) return FDC_ERR_SHAPE;
