@@ -132,9 +132,9 @@ int fdc_plan_graph(const fdc_graph_desc* g, fdc_plan** out)
         p->sm_count = prop.multiProcessorCount;
         e = cudaMalloc((void**)&p->d, sizeof(PlanDev));
     }
-    if (e == cudaSuccess) e = cudaMalloc((void**)&p->d_status, (4 + FDC_PAIR_COUNTERS) * sizeof(int32_t));
+    if (e == cudaSuccess) e = cudaMalloc((void**)&p->d_status, (4 + FDC_PAIR_COUNTERS + 2 * FDC_MEMO_INTS) * sizeof(int32_t));
     if (e == cudaSuccess) e = cudaMemcpy(p->d, &p->h, sizeof(PlanDev), cudaMemcpyHostToDevice);
-    if (e == cudaSuccess) e = cudaMemset(p->d_status, 0, (4 + FDC_PAIR_COUNTERS) * sizeof(int32_t));
+    if (e == cudaSuccess) e = cudaMemset(p->d_status, 0, (4 + FDC_PAIR_COUNTERS + 2 * FDC_MEMO_INTS) * sizeof(int32_t));
     if (e != cudaSuccess) {
         int rc = set_cuda_error(e);
         fdc_plan_destroy(p);
@@ -142,6 +142,8 @@ int fdc_plan_graph(const fdc_graph_desc* g, fdc_plan** out)
     }
     p->d_ticket = p->d_status + 2;
     p->d_pair_cnt = p->d_status + 4;
+    p->d_split_memo = p->d_pair_cnt + FDC_PAIR_COUNTERS;
+    p->attn_seq = 0;
     *out = p;
     return FDC_OK;
 }

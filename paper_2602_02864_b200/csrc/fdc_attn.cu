@@ -161,12 +161,17 @@ int fdc_decode_attn(const fdc_plan* p, const fdc_kv_desc* kv, int32_t layer, con
     }
     rc = FDC_ERR_SHAPE;
     a.pair_cnt = nullptr;
+    a.split_memo = nullptr;
+    a.seq = 0;
     bool fused = false;                 // the split kernel merged the partials itself
     if (kv->dtype == FDC_BF16 && (p->attn_kernel == 0 || p->attn_kernel == 3)) {
         if ((long long)kv->batch * kv->hkv <= FDC_PAIR_COUNTERS) a.pair_cnt = p->d_pair_cnt;
+        a.split_memo = (a.pair_cnt && kv->batch <= FDC_MEMO_BATCH && a.n_cta <= FDC_MEMO_CTAS) ? p->d_split_memo : nullptr;
+        a.seq = ++const_cast<fdc_plan*>(p)->attn_seq;       // calls on one plan are ordered (see fdc.h)
         rc = launch_attn_tc(a, kv->head_dim, st);
         fused = rc == FDC_OK && a.pair_cnt != nullptr;
         a.pair_cnt = nullptr;
+        a.split_memo = nullptr;
     }
     if (kv->dtype == FDC_BF16 && (p->attn_kernel == 2 || (rc == FDC_ERR_SHAPE && p->attn_kernel != 1)))
         rc = launch_attn_mma(a, kv->head_dim, st);

@@ -1190,6 +1190,27 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, con
     cx.abortp = &abort_flag;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // After a layer's 270 MB of KV went through the memory system, the address translations of the
+    // small arrays are gone, and the first access to each costs a page walk (microseconds).  Eight
+    // threads touch them now: the walks run side by side and overlap the set-up below and the wait
+    // for the kernel before this one.  The values are not used (that kernel may still be running).
+    if (threadIdx.x >= 32 && threadIdx.x < 40) {
+        const void* a;
+        switch (threadIdx.x - 32) {
+            case 0: a = p.n_active; break;
+            case 1: a = p.ntiles; break;
+            case 2: a = p.split_memo ? p.split_memo + ((p.seq - 1u) & 1u) * FDC_MEMO_INTS : nullptr; break;
+            case 3: a = p.split_memo ? p.split_memo + ((p.seq - 1u) & 1u) * FDC_MEMO_INTS + FDC_MEMO_ENTRIES + 4 * blockIdx.x : nullptr; break;
+            case 4: a = p.tiles; break;
+            case 5: a = p.q; break;
+            case 6: a = p.mask; break;
+            default: a = p.out; break;
+        }
+        if (a) {
+            uint32_t unused;
+            asm volatile("ld.global.cg.b32 %0, [%1];" : "=r"(unused) : "l"(a) : "memory");
+        }
+    }
     if (threadIdx.x == 0) abort_flag = 0;
     if (threadIdx.x < 4) cx.rflag[threadIdx.x] = -1;
     // ---- set-up that needs no global memory: barriers, TMEM
@@ -1231,13 +1252,71 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, con
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     bool active = true;                       // this CTA has units (uniform over the CTA)
     long long lo = 0, hi = 0;
-    for (int i = threadIdx.x; i < p.batch; i += THREADS) cx.nact[i] = p.n_active[i];
-    const long long total = scan_ntiles(p.ntiles, p.batch, cx.pre);
+    // The layers of one forward pass see the same per-scene counts, so the previous launch on this
+    // plan has left its work split in the memo, with the counts it was computed from.  Its loads
+    // are issued first; they are in flight together with those of the counts.
+    constexpr int MEMO_MAGIC = 0x5D170000 | (W_MASKED << 8) | W_PAIR;
+    const int32_t* mrd = p.split_memo ? p.split_memo + ((p.seq - 1u) & 1u) * FDC_MEMO_INTS : nullptr;
+    int4 mh0 = make_int4(0, 0, 0, 0), mh1 = mh0, mh2 = mh0, me = mh0;
+    int m_na = -1, m_nt = -1, m_prev = 0;
+    if (mrd) {
+        mh0 = __ldcg(reinterpret_cast<const int4*>(mrd));
+        mh1 = __ldcg(reinterpret_cast<const int4*>(mrd) + 1);
+        mh2 = __ldcg(reinterpret_cast<const int4*>(mrd) + 2);
+        me = __ldcg(reinterpret_cast<const int4*>(mrd + FDC_MEMO_ENTRIES) + blockIdx.x);
+        if ((int)threadIdx.x < p.batch) {
+            m_na = __ldcg(mrd + 16 + threadIdx.x);
+            m_nt = __ldcg(mrd + 16 + FDC_MEMO_BATCH + threadIdx.x);
+        }
+        if ((int)threadIdx.x <= p.batch) m_prev = __ldcg(mrd + 16 + 2 * FDC_MEMO_BATCH + threadIdx.x);
+    }
+    // the counts: every load is issued before the first use, so that all of them (and the memo's)
+    // share one trip to memory; the raw tile counts wait in prev[] for the scan
+    {
+        int na[4], nt[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int i = threadIdx.x + j * THREADS;
+            na[j] = i < p.batch ? p.n_active[i] : 0;
+            nt[j] = i < p.batch ? p.ntiles[i] : 0;
+        }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int i = threadIdx.x + j * THREADS;
+            if (i < p.batch) {
+                cx.nact[i] = na[j];
+                cx.prev[i] = nt[j];
+            }
+        }
+        for (int i = threadIdx.x + 4 * THREADS; i < p.batch; i += THREADS) {
+            cx.nact[i] = p.n_active[i];
+            cx.prev[i] = p.ntiles[i];
+        }
+    }
+    __syncthreads();
+    const long long total = scan_ntiles(cx.prev, p.batch, cx.pre);
     const long long U = total * p.hkv;
     if (U == 0) active = false;
     cx.tpart = 0;
     cx.n_cta = p.n_cta;
-    if (!active) {
+    cx.vtot = 0;
+    cx.npre = p.P / TILE;
+    bool hit = false;
+    if (mrd) {
+        int same = mh0.x == MEMO_MAGIC && mh0.y == (int)(p.seq - 1u) && mh0.z == p.hkv && mh0.w == p.n_cta && mh1.x == p.P && mh1.y == p.batch;
+        if ((int)threadIdx.x < p.batch) same = same && m_na == cx.nact[threadIdx.x] && m_nt == cx.pre[threadIdx.x + 1] - cx.pre[threadIdx.x];
+        hit = __syncthreads_and(same) != 0;
+    }
+    if (hit) {
+        // same counts as the launch before: its split stands
+        cx.tpart = mh1.z;
+        cx.n_cta = mh1.w;
+        cx.vtot = ((long long)mh2.y << 32) | (uint32_t)mh2.x;
+        if ((int)threadIdx.x <= p.batch) cx.prev[threadIdx.x] = m_prev;
+        __syncthreads();
+        lo = ((long long)me.y << 32) | (uint32_t)me.x;
+        hi = ((long long)me.w << 32) | (uint32_t)me.z;
+    } else if (!active) {
     } else if (p.pair_cnt) {
         // This kernel also merges the partial results of a pair.  Ending one pair and starting the
         // next inside a CTA costs as much as streaming a dozen tiles (drain, partial write, merge,
@@ -1342,6 +1421,25 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, con
         hi = cta_first_unit(blockIdx.x + 1, U, cx.n_cta);
     }
     if (lo >= hi || (int)blockIdx.x >= cx.n_cta) active = false;
+    if (p.split_memo) {
+        // leave the split to the next launch (plain stores, nobody waits for them)
+        int32_t* mwr = p.split_memo + (p.seq & 1u) * FDC_MEMO_INTS;
+        if (threadIdx.x == 0)
+            reinterpret_cast<int4*>(mwr + FDC_MEMO_ENTRIES)[blockIdx.x] =
+                active ? make_int4((int)(uint32_t)lo, (int)(lo >> 32), (int)(uint32_t)hi, (int)(hi >> 32)) : make_int4(0, 0, 0, 0);
+        if (blockIdx.x == 0) {
+            if (threadIdx.x == 0) {
+                reinterpret_cast<int4*>(mwr)[0] = make_int4(MEMO_MAGIC, (int)p.seq, p.hkv, p.n_cta);
+                reinterpret_cast<int4*>(mwr)[1] = make_int4(p.P, p.batch, cx.tpart, cx.n_cta);
+                reinterpret_cast<int4*>(mwr)[2] = make_int4((int)(uint32_t)cx.vtot, (int)(cx.vtot >> 32), 0, 0);
+            }
+            if ((int)threadIdx.x < p.batch) {
+                mwr[16 + threadIdx.x] = cx.nact[threadIdx.x];
+                mwr[16 + FDC_MEMO_BATCH + threadIdx.x] = cx.pre[threadIdx.x + 1] - cx.pre[threadIdx.x];
+            }
+            if ((int)threadIdx.x <= p.batch) mwr[16 + 2 * FDC_MEMO_BATCH + threadIdx.x] = U > 0 ? cx.prev[threadIdx.x] : 0;
+        }
+    }
 
     if (!active) {
     } else if (warp == W_PROD) {

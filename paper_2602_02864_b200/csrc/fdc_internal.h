@@ -7,6 +7,15 @@
 #include "fdc.h"
 
 #define FDC_PAIR_COUNTERS 65536
+// Work-split memo of the tcgen05 attention kernel: the layers of one forward pass see the same
+// per-scene counts, so the split of one launch is kept (with the counts it was computed from) and
+// the next launch only checks that the counts are unchanged.  Layout of a slot, in int32:
+// [0..15] header, [16..) n_active[FDC_MEMO_BATCH], tiles[FDC_MEMO_BATCH], prev[FDC_MEMO_BATCH + 1],
+// [FDC_MEMO_ENTRIES..) first and last unit of each CTA (2 x int64).
+#define FDC_MEMO_BATCH 256
+#define FDC_MEMO_CTAS 256
+#define FDC_MEMO_ENTRIES 800
+#define FDC_MEMO_INTS (FDC_MEMO_ENTRIES + 4 * FDC_MEMO_CTAS)
 
 namespace fdc {
 
@@ -43,6 +52,8 @@ struct fdc_plan {
     int32_t*      d_status;          // sticky FDC_DEV_* bits
     int32_t*      d_ticket;          // [2] scratch of the frontier kernel's cross-block reduction
     int32_t*      d_pair_cnt;        // [FDC_PAIR_COUNTERS] arrivals per (scene, KV head) of the fused combine (zero between calls)
+    int32_t*      d_split_memo;      // [2][FDC_MEMO_INTS] work split of the last attention launch and the counts it was made from
+    uint32_t      attn_seq;          // attention launches on this plan so far (selects the memo slot)
     int           device;
     int           sm_count;
     int           attn_kernel;       // 0 auto
@@ -71,6 +82,8 @@ struct AttnParams {
     float           scale_log2;      // softmax scale * log2(e)
     int32_t*        status;          // sticky FDC_DEV_* bits
     int32_t*        pair_cnt;        // per (scene, KV head) arrival counters: the split kernel also combines (nullptr: it does not)
+    int32_t*        split_memo;      // [2][FDC_MEMO_INTS] (nullptr: the work split is always computed)
+    uint32_t        seq;             // number of this launch on the plan
 };
 
 extern int64_t g_launches;

@@ -12,32 +12,55 @@ using namespace fdc;
 
 namespace {
 
-// grid.x = batch * max_active (one block per branch slot); threads copy 16-byte vectors.
-__global__ void kv_append_kernel(char* __restrict__ k, char* __restrict__ v, int64_t stride_scene_b,
+// One block per branch slot, or a grid-stride loop over the slots when there are more slots than
+// blocks; threads copy 16-byte vectors.
+__global__ void __launch_bounds__(128) kv_append_kernel(char* __restrict__ k, char* __restrict__ v, int64_t stride_scene_b,
                                  int64_t stride_head_b, int64_t stride_row_b, int rows, int hkv, int row_bytes,
-                                 int max_active, const int32_t* __restrict__ n_active,
+                                 int max_active, int n_slots, const int32_t* __restrict__ n_active,
                                  const int32_t* __restrict__ kv_row, const char* __restrict__ k_new,
                                  const char* __restrict__ v_new, int32_t* __restrict__ status)
 {
-    // programmatic dependent launch (see the attention kernel): wait for the kernel before this one,
-    // let the one after it be scheduled
-    asm volatile("griddepcontrol.wait;" ::: "memory");
+    // Programmatic dependent launch.  The kernel after this one (the attention kernel) may be
+    // scheduled as soon as every block of this grid is resident: its blocks then take the SMs as
+    // they become free, set themselves up and wait for this grid to complete.  This grid waits for
+    // the kernel before it, so completion still follows the stream order.  The grid is small
+    // (at most n_slots blocks of 128 threads and few registers) so that all of it is resident early.
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    const int s = blockIdx.x / max_active, b = blockIdx.x - s * max_active;
-    if (b >= n_active[s]) return;
-    const int row = kv_row[blockIdx.x];
-    if (row < 0 || row >= rows) {
-        if (threadIdx.x == 0) atomicOr(status, FDC_DEV_ROW_RANGE);
-        return;
-    }
-    const int vec_per_row = row_bytes >> 4;
-    const size_t src0 = (size_t)blockIdx.x * hkv * row_bytes;
-    for (int i = threadIdx.x; i < hkv * vec_per_row; i += blockDim.x) {
-        const int g = i / vec_per_row, c = i - g * vec_per_row;
-        const size_t src = src0 + (size_t)g * row_bytes + (size_t)c * 16;
-        const size_t dst = (size_t)s * stride_scene_b + (size_t)g * stride_head_b + (size_t)row * stride_row_b + (size_t)c * 16;
-        *reinterpret_cast<uint4*>(k + dst) = *reinterpret_cast<const uint4*>(k_new + src);
-        *reinterpret_cast<uint4*>(v + dst) = *reinterpret_cast<const uint4*>(v_new + src);
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    // All loads of a slot are issued before anything depends on them (the rows of idle branch
+    // slots exist in k_new / v_new too, so they can be read before n_active is known): one trip
+    // to memory instead of three in a row.
+    const int vec_per_row = row_bytes >> 4, nvec = hkv * vec_per_row;
+    for (int slot = blockIdx.x; slot < n_slots; slot += gridDim.x) {
+        const int s = slot / max_active, b = slot - s * max_active;
+        const size_t src0 = (size_t)slot * hkv * row_bytes;
+        const int na = n_active[s];
+        const int row = kv_row[slot];
+        for (int i0 = threadIdx.x; i0 < nvec; i0 += 2 * blockDim.x) {
+            const int i1 = i0 + blockDim.x;
+            uint4 kk[2], vv[2];
+            kk[0] = *reinterpret_cast<const uint4*>(k_new + src0 + (size_t)i0 * 16);
+            vv[0] = *reinterpret_cast<const uint4*>(v_new + src0 + (size_t)i0 * 16);
+            if (i1 < nvec) {
+                kk[1] = *reinterpret_cast<const uint4*>(k_new + src0 + (size_t)i1 * 16);
+                vv[1] = *reinterpret_cast<const uint4*>(v_new + src0 + (size_t)i1 * 16);
+            }
+            if (b >= na) break;
+            if (row < 0 || row >= rows) {
+                if (threadIdx.x == 0) atomicOr(status, FDC_DEV_ROW_RANGE);
+                break;
+            }
+#pragma unroll
+            for (int j = 0; j < 2; ++j) {
+                const int i = j ? i1 : i0;
+                if (i < nvec) {
+                    const int g = i / vec_per_row, c = i - g * vec_per_row;
+                    const size_t dst = (size_t)s * stride_scene_b + (size_t)g * stride_head_b + (size_t)row * stride_row_b + (size_t)c * 16;
+                    *reinterpret_cast<uint4*>(k + dst) = kk[j];
+                    *reinterpret_cast<uint4*>(v + dst) = vv[j];
+                }
+            }
+        }
     }
 }
 
@@ -78,10 +101,13 @@ extern "C" int fdc_kv_append(const fdc_plan* p, const fdc_kv_desc* kv, int32_t l
     char* vb = (char*)kv->v + (size_t)layer * kv->stride_layer * es;
     const int row_bytes = kv->head_dim * es;
     int threads = kv->hkv * (row_bytes >> 4);
-    threads = threads > 256 ? 256 : ((threads + 31) & ~31);
+    const int n_slots = kv->batch * p->h.max_active;
+    // blocks small enough to sit beside a resident attention block: one of 128 threads per SM, or two of 64
+    const int per_sm = n_slots > p->sm_count ? 2 : 1;
+    threads = threads > 128 / per_sm ? 128 / per_sm : ((threads + 31) & ~31);
     {
         cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3(kv->batch * p->h.max_active);
+        cfg.gridDim = dim3(n_slots < per_sm * p->sm_count ? n_slots : per_sm * p->sm_count);
         cfg.blockDim = dim3(threads);
         cfg.dynamicSmemBytes = 0;
         cfg.stream = (cudaStream_t)stream;
@@ -91,7 +117,7 @@ extern "C" int fdc_kv_append(const fdc_plan* p, const fdc_kv_desc* kv, int32_t l
         cfg.attrs = at;
         cfg.numAttrs = 1;
         FDC_CUDA(cudaLaunchKernelEx(&cfg, kv_append_kernel, kb, vb, (int64_t)(kv->stride_scene * es), (int64_t)(kv->stride_head * es),
-                                    (int64_t)(kv->stride_row * es), (int)kv->rows, (int)kv->hkv, row_bytes, (int)p->h.max_active, d_n_active,
+                                    (int64_t)(kv->stride_row * es), (int)kv->rows, (int)kv->hkv, row_bytes, (int)p->h.max_active, n_slots, d_n_active,
                                     d_kv_row, (const char*)d_k_new, (const char*)d_v_new, p->d_status));
     }
     note_launch();
