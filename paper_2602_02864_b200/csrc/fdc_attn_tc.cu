@@ -1190,27 +1190,6 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, con
     cx.abortp = &abort_flag;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    // After a layer's 270 MB of KV went through the memory system, the address translations of the
-    // small arrays are gone, and the first access to each costs a page walk (microseconds).  Eight
-    // threads touch them now: the walks run side by side and overlap the set-up below and the wait
-    // for the kernel before this one.  The values are not used (that kernel may still be running).
-    if (threadIdx.x >= 32 && threadIdx.x < 40) {
-        const void* a;
-        switch (threadIdx.x - 32) {
-            case 0: a = p.n_active; break;
-            case 1: a = p.ntiles; break;
-            case 2: a = p.split_memo ? p.split_memo + ((p.seq - 1u) & 1u) * FDC_MEMO_INTS : nullptr; break;
-            case 3: a = p.split_memo ? p.split_memo + ((p.seq - 1u) & 1u) * FDC_MEMO_INTS + FDC_MEMO_ENTRIES + 4 * blockIdx.x : nullptr; break;
-            case 4: a = p.tiles; break;
-            case 5: a = p.q; break;
-            case 6: a = p.mask; break;
-            default: a = p.out; break;
-        }
-        if (a) {
-            uint32_t unused;
-            asm volatile("ld.global.cg.b32 %0, [%1];" : "=r"(unused) : "l"(a) : "memory");
-        }
-    }
     if (threadIdx.x == 0) abort_flag = 0;
     if (threadIdx.x < 4) cx.rflag[threadIdx.x] = -1;
     // ---- set-up that needs no global memory: barriers, TMEM
