@@ -174,7 +174,9 @@ int fdc_build_masks(const fdc_plan* plan, int32_t batch, const void* d_state, ui
 /* Sec. 3.3 (shared KV cache, reused by all later passes): for every scene s and branch
  * b < d_n_active[s], copy d_k_new/d_v_new [batch][max_active][hkv][head_dim] into cache row
  * d_kv_row[s][b] of `layer`.  Padding rows are never written.  Rows outside [0, rows) are
- * skipped and flagged in the plan's status word. */
+ * skipped and flagged in the plan's status word.  d_k_new, d_v_new and d_kv_row are read for
+ * every branch slot, idle ones included (the loads are issued before d_n_active is known), so
+ * all of [batch][max_active] must be addressable; what idle slots hold does not matter. */
 int fdc_kv_append(const fdc_plan* plan, const fdc_kv_desc* kv, int32_t layer, const int32_t* d_n_active,
                   const int32_t* d_kv_row, const void* d_k_new, const void* d_v_new, void* stream);
 
@@ -192,8 +194,9 @@ int fdc_attn_workspace_bytes(const fdc_plan* plan, const fdc_kv_desc* kv, size_t
  * may hold anything (NaN included).  d_workspace: DEVICE, 256-byte aligned,
  * >= fdc_attn_workspace_bytes; its contents are undefined afterwards.
  * The tcgen05 kernel merges its split partials itself and keeps per-(scene, KV head) arrival
- * counters in the plan: calls that use the same plan must be ordered on the GPU (one stream, or
- * events); use one plan per concurrently decoding batch. */
+ * counters in the plan, and it leaves its work split there for the next call (checked against
+ * d_n_active / d_ntiles before it is reused): calls that use the same plan must be ordered on
+ * the GPU (one stream, or events); use one plan per concurrently decoding batch. */
 int fdc_decode_attn(const fdc_plan* plan, const fdc_kv_desc* kv, int32_t layer, const int32_t* d_n_active,
                     const uint64_t* d_mask, const int32_t* d_tiles, const int32_t* d_ntiles,
                     const void* d_q, void* d_out, float scale, void* d_workspace, size_t ws_bytes,
