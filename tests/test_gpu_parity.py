@@ -193,3 +193,47 @@ def test_softmax_reference_is_raised_when_scores_jump(monkeypatch):
         w = wl.cfg4_sweep(2048, branches, 2)
         r = run_and_compare(w, check_steps={0, 1, 2, 33, 63}, kernel=3)
         assert r["checked"] > 0
+
+
+def test_work_split_of_the_previous_call_is_reused_only_for_the_same_counts():
+    """The attention kernel keeps its work split in the plan for the next call and reuses it
+    when n_active and ntiles are unchanged.  A repeated call must give the same bits; a call
+    with other counts (one scene switched off) must not use the stale split; and going back
+    to the first counts must reproduce the first result."""
+    from paper_2602_02864_b200 import fdc
+    from harness import alloc_cache, write_prefix, BF16_MAX_ABS, f32
+    w = wl.cfg2_batched(layers=1, batch=4)
+    dev = "cuda"
+    sess = fdc.DecodeSession(w.n_nodes, w.edges, w.slot_cap, w.n_fixed, w.prefix_len, w.max_active, w.batch, dev)
+    k, v = alloc_cache(w, dev)
+    write_prefix(w, k, v)
+    sess.bind_cache(k, v, w.hq)
+    sess.init(torch.from_numpy(w.lens).to(dev))
+    sess.frontier(None)
+    sess.build_masks()
+    q, kn, vn = wl.step_qkv(w, 0, 0, dev)
+    sess.kv_append(0, kn, vn)
+
+    def attend(n_active, ntiles):
+        out = torch.full_like(q, 7.0)
+        fdc.fdc_decode_attn(sess.plan, sess.kv, 0, n_active, sess.mask, sess.tiles, ntiles, q, out, w.softmax_scale,
+                            sess.workspace, sess.ws_bytes)
+        torch.cuda.synchronize()
+        return out
+
+    first = attend(sess.n_active, sess.ntiles)            # split computed
+    again = attend(sess.n_active, sess.ntiles)            # same counts: split reused
+    assert torch.equal(first, again)
+    assert np.isfinite(f32(first)[sess.n_active.cpu().numpy().nonzero()[0], 0]).all()
+    na2, nt2 = sess.n_active.clone(), sess.ntiles.clone()
+    na2[1] = 0                                            # scene 1 has finished: no branch, no tile
+    nt2[1] = 0
+    other = attend(na2, nt2)
+    assert bool((other[1] == 7.0).all())                  # nothing written for the scene that is off
+    for s in (0, 2, 3):                                   # the others: same result up to the other split's rounding
+        A = int(sess.n_active[s])
+        assert np.abs(f32(other[s, :A]) - f32(first[s, :A])).max() <= BF16_MAX_ABS
+    back = attend(sess.n_active, sess.ntiles)
+    assert torch.equal(first, back)
+    assert sess.status() == 0
+    sess.close()
