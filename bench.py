@@ -53,6 +53,7 @@ def log(*a):
     print(*a, file=sys.stderr, flush=True)
 
 
+FUSED_APPEND = True         # fdc_set_fused_append: one kernel per layer (--separate-append: two)
 LAYERS_OVERRIDE = None      # --layers: fewer layers of the same configuration (profiling captures)
 
 
@@ -146,6 +147,8 @@ class StepBench:
                 t[:, l, :, :w.prefix_len] = (torch.randn((w.batch, w.hkv, w.prefix_len, w.head_dim), generator=g,
                                                          device=device) * w.kv_scale).to(w.torch_dtype)
         self.sess.bind_cache(self.k, self.v, w.hq)
+        if FUSED_APPEND:
+            self.sess.set_fused_append(True)
         self.lens = torch.from_numpy(w.lens).to(device)
         qs = (n_steps, w.layers, w.batch, w.max_active, w.hq, w.head_dim)
         ks = (n_steps, w.layers, w.batch, w.max_active, w.hkv, w.head_dim)
@@ -250,6 +253,23 @@ def run_fdc(args, rank: int, world: int):
         ms = replicas.max_over_ranks(e0.elapsed_time(e1), device)      # the job's time: the slowest replica
         replicas.barrier()
 
+        # pass 1b (context only): the same steps with kv_append as a kernel of its own
+        ms_separate = None
+        if FUSED_APPEND and world == 1:
+            sb.sess.set_fused_append(False)
+            sb.reset()
+            for i in range(W):
+                sb.step(i)
+            torch.cuda.synchronize()
+            e0, e1 = ev(), ev()
+            e0.record(stream)
+            for i in range(W, total):
+                sb.step(i)
+            e1.record(stream)
+            torch.cuda.synchronize()
+            ms_separate = e0.elapsed_time(e1)
+            sb.sess.set_fused_append(True)
+
         # pass 2: per-launch duration of the dominant kernel (split-KV pass), CUDA events recorded by
         # the library itself on the launching stream around every such launch of the same K steps
         sb.reset()
@@ -315,6 +335,7 @@ def run_fdc(args, rank: int, world: int):
         res = {"workload": name, "value": value, "ms": ms, "ms_per_step": ms / K, "launches": launches,
                "roofline": roof, "e2e": e2e, "clocks": clocks, "status": status,
                "step_us": round(ms / K * 1e3, 1), "layer_step_us": round(ms / K / w.layers * 1e3, 2),
+               "layer_step_us_separate_append": None if ms_separate is None else round(ms_separate / K / w.layers * 1e3, 2),
                "bytes_per_step": int(timed_bytes / K), "avg_active_per_scene": float(sb.nact_log[W:].float().mean()),
                "pct_of_8TBs": round(100 * value / world / NOMINAL_HBM_GBS, 1),
                "pct_of_measured_copy": round(100 * value / world / peak, 1)}
@@ -331,7 +352,7 @@ def run_fdc(args, rank: int, world: int):
                 continue
             r, _ = measure(other, min(args.steps, 20), max(3, min(args.warmup, 5)), False, False)
             also[other] = {k: (round(v, 2) if isinstance(v, float) else v) for k, v in r.items()
-                           if k in ("value", "step_us", "layer_step_us", "bytes_per_step", "pct_of_8TBs",
+                           if k in ("value", "step_us", "layer_step_us", "layer_step_us_separate_append", "bytes_per_step", "pct_of_8TBs",
                                     "pct_of_measured_copy", "roofline", "avg_active_per_scene")}
             also[other]["workload"] = WORKLOAD_TEXT[other]
 
@@ -348,8 +369,12 @@ def run_fdc(args, rank: int, world: int):
                        "l2": "inputs larger than L2: each layer reads its own KV buffer, %.1f GB of KV per step"
                              % (main["bytes_per_step"] / 1e9),
                        "parallelism": "replicas" if world > 1 else "1 GPU",
-                       "step": "frontier + build_masks + layers x (kv_append + decode_attn[split-KV pass with the combine fused in])"},
+                       "step": ("frontier + build_masks + layers x (kv_append recorded, carried out inside decode_attn "
+                                "[fdc_set_fused_append]: one kernel that appends, runs the split-KV pass and combines)")
+                               if FUSED_APPEND else
+                               "frontier + build_masks + layers x (kv_append + decode_attn[split-KV pass with the combine fused in])"},
             "step_us": main["step_us"], "layer_step_us": main["layer_step_us"],
+            "layer_step_us_separate_append": main["layer_step_us_separate_append"],
             "bytes_per_step": main["bytes_per_step"], "avg_active_branches_per_scene": round(main["avg_active_per_scene"], 2),
             "pct_of_8TBs": main["pct_of_8TBs"], "pct_of_measured_copy": main["pct_of_measured_copy"],
             "roofline": main["roofline"], "cpu_baseline": cpu, "e2e": main["e2e"], "clocks": main["clocks"],
@@ -420,11 +445,15 @@ def main():
     ap.add_argument("--impl", default="fdc", choices=["fdc", "reference"])
     ap.add_argument("--no-also", action="store_true", help="skip the short runs of the other configurations")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU baseline leg")
+    ap.add_argument("--separate-append", action="store_true",
+                    help="launch kv_append as a kernel of its own instead of inside the attention kernel")
     ap.add_argument("--layers", type=int, default=None,
                     help="run only this many layers of the configuration (small ncu captures; not a bench number)")
     args = ap.parse_args()
     global LAYERS_OVERRIDE
     LAYERS_OVERRIDE = args.layers
+    global FUSED_APPEND
+    FUSED_APPEND = not args.separate_append
     rank = int(os.environ.get("RANK", 0))
     world = int(os.environ.get("WORLD_SIZE", 1))
     if args.impl == "reference":

@@ -245,6 +245,21 @@ int fdc_status(const fdc_plan* plan, int32_t* host_bits, int32_t clear, void* st
 int fdc_set_attn_kernel(fdc_plan* plan, int32_t which);
 const char* fdc_kernel_name(int32_t which);
 
+/* Fused append (off by default; Sec. 3.3's shared cache, written and read in one kernel).  While
+ * on, an fdc_kv_append on this plan whose cache the tcgen05 attention kernel serves (bf16,
+ * head_dim 128) launches nothing: its arguments are recorded, and the NEXT fdc_decode_attn for
+ * the same cache, layer, stream and d_n_active writes the rows inside its own kernel, each by
+ * the thread block that owns the row's KV tile, before that block loads the tile.  One kernel
+ * per layer instead of two dependent ones.  Until that call returns the caller must not read
+ * the rows from the cache, and must leave d_n_active, d_kv_row, d_k_new and d_v_new as they
+ * were.  Any other call on the plan (another append, an attention call that does not match,
+ * fdc_frontier, fdc_build_masks, fdc_state_init, fdc_status, fdc_set_*, fdc_plan_destroy)
+ * first launches the recorded append on its own, so no append is ever lost.  Differences from
+ * the separate kernel: rows below prefix_len are refused (flagged FDC_DEV_ROW_RANGE like rows
+ * >= rows), and a row is written only if its tile is in d_tiles (fdc_build_masks lists it: a
+ * new token sees itself). */
+int fdc_set_fused_append(fdc_plan* plan, int32_t on);
+
 /* Instrumentation for benchmarks: while enabled, fdc_decode_attn records CUDA events on the
  * launching stream before its split pass, between the passes and after its combine pass (not
  * usable during stream capture).  fdc_profile_read waits for the recorded events, returns

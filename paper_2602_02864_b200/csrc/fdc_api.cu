@@ -144,6 +144,8 @@ int fdc_plan_graph(const fdc_graph_desc* g, fdc_plan** out)
     p->d_pair_cnt = p->d_status + 4;
     p->d_split_memo = p->d_pair_cnt + FDC_PAIR_COUNTERS;
     p->attn_seq = 0;
+    p->fuse_append = 0;
+    p->pend.valid = 0;
     *out = p;
     return FDC_OK;
 }
@@ -151,6 +153,7 @@ int fdc_plan_graph(const fdc_graph_desc* g, fdc_plan** out)
 int fdc_plan_destroy(fdc_plan* p)
 {
     if (!p) return FDC_ERR_NULL;
+    flush_pending_append(p);              // a recorded append is still owed to the cache
     prof_destroy(p);
     if (p->d) cudaFree(p->d);
     if (p->d_status) cudaFree(p->d_status);
@@ -221,6 +224,10 @@ int fdc_plan_critical_path(const fdc_plan* p, const int32_t* len, int32_t* steps
 int fdc_status(const fdc_plan* p, int32_t* host_bits, int32_t clear, void* stream)
 {
     if (!p || !host_bits) return FDC_ERR_NULL;
+    {
+        int rcf = flush_pending_append(p);
+        if (rcf) return rcf;
+    }
     cudaStream_t st = (cudaStream_t)stream;
     FDC_CUDA(cudaMemcpyAsync(host_bits, p->d_status, sizeof(int32_t), cudaMemcpyDeviceToHost, st));
     if (clear) {

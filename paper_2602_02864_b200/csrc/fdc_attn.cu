@@ -46,6 +46,14 @@ void prof_destroy(fdc_plan* p)
     delete pr;
     p->prof = nullptr;
 }
+
+// The conditions under which fdc_decode_attn runs the tcgen05 kernel with the combine fused in
+// (the only kernel that can also carry out a recorded append).
+bool takes_tc_kernel(const fdc_plan* p, const fdc_kv_desc* kv)
+{
+    return kv->dtype == FDC_BF16 && kv->head_dim == 128 && (p->attn_kernel == 0 || p->attn_kernel == 3) &&
+           (long long)p->h.max_active * (kv->hq / kv->hkv) <= 128 && (long long)kv->batch * kv->hkv <= FDC_PAIR_COUNTERS;
+}
 }  // namespace fdc
 
 extern "C" {
@@ -88,8 +96,21 @@ int fdc_attn_workspace_bytes(const fdc_plan* p, const fdc_kv_desc* kv, size_t* b
     return FDC_OK;
 }
 
+int fdc_set_fused_append(fdc_plan* p, int32_t on)
+{
+    if (!p) return FDC_ERR_NULL;
+    int rc = flush_pending_append(p);
+    if (rc) return rc;
+    p->fuse_append = on ? 1 : 0;
+    return FDC_OK;
+}
+
 int fdc_set_attn_kernel(fdc_plan* p, int32_t which)
 {
+    if (p) {
+        int rcf = flush_pending_append(p);
+        if (rcf) return rcf;
+    }
     if (!p) return FDC_ERR_NULL;
     if (which < 0 || which > 3) return FDC_ERR_RANGE;
     p->attn_kernel = which;
@@ -118,6 +139,19 @@ int fdc_decode_attn(const fdc_plan* p, const fdc_kv_desc* kv, int32_t layer, con
     if (((uintptr_t)d_q & 15) || ((uintptr_t)d_out & 15)) return FDC_ERR_SHAPE;
     if (!(scale > 0.f) || !std::isfinite(scale)) return FDC_ERR_RANGE;
     const int es = kv->dtype == FDC_F32 ? 4 : 2;
+    // a recorded append is carried out by this call's kernel if it belongs to it, else on its own first
+    fdc_pending_append app = p->pend;
+    if (app.valid) {
+        const bool mine = takes_tc_kernel(p, kv) && app.kv.k == kv->k && app.kv.v == kv->v && app.layer == layer &&
+                          app.stream == stream && app.d_n_active == d_n_active && app.kv.stride_layer == kv->stride_layer;
+        if (mine) {
+            const_cast<fdc_plan*>(p)->pend.valid = 0;
+        } else {
+            rc = flush_pending_append(p);
+            if (rc) return rc;
+            app.valid = 0;
+        }
+    }
 
     AttnParams a;
     a.k = (const char*)kv->k + (size_t)layer * kv->stride_layer * es;
@@ -147,6 +181,8 @@ int fdc_decode_attn(const fdc_plan* p, const fdc_kv_desc* kv, int32_t layer, con
     a.ws_ml = a.ws_o + slots * a.mmax * kv->head_dim;
     a.n_cta = p->sm_count;
     a.status = p->d_status;
+    a.app_row = nullptr;
+    a.app_k = a.app_v = nullptr;
 
     cudaStream_t st = (cudaStream_t)stream;
     Prof* pr = p->prof_on ? (Prof*)p->prof : nullptr;
@@ -168,7 +204,18 @@ int fdc_decode_attn(const fdc_plan* p, const fdc_kv_desc* kv, int32_t layer, con
         if ((long long)kv->batch * kv->hkv <= FDC_PAIR_COUNTERS) a.pair_cnt = p->d_pair_cnt;
         a.split_memo = (a.pair_cnt && kv->batch <= FDC_MEMO_BATCH && a.n_cta <= FDC_MEMO_CTAS) ? p->d_split_memo : nullptr;
         a.seq = ++const_cast<fdc_plan*>(p)->attn_seq;       // calls on one plan are ordered (see fdc.h)
+        if (app.valid) {
+            a.app_row = app.d_kv_row;
+            a.app_k = app.d_k_new;
+            a.app_v = app.d_v_new;
+        }
         rc = launch_attn_tc(a, kv->head_dim, st);
+        a.app_row = nullptr;
+        if (app.valid && rc != FDC_OK) {
+            // the kernel that would have written the rows was not launched: append on its own after all
+            int rca = launch_kv_append(p, kv, layer, app.d_n_active, app.d_kv_row, app.d_k_new, app.d_v_new, stream);
+            if (rca) return rca;
+        }
         fused = rc == FDC_OK && a.pair_cnt != nullptr;
         a.pair_cnt = nullptr;
         a.split_memo = nullptr;

@@ -178,7 +178,7 @@ __device__ __forceinline__ float ord_to(int i) { return __int_as_float(i ^ ((i >
 
 // Everything a role needs to find its barriers and buffers.
 struct Ctx {
-    uint32_t k_full, k_empty, v_full, v_empty, v_clean, s_full, s_free, p_full, pv_done, q_ready, o_free;
+    uint32_t k_full, k_empty, v_full, v_empty, v_clean, s_full, s_free, p_full, pv_done, q_ready, o_free, app_done;
     int ns, s_stride;                // S^T buffers in TMEM (4 of 64 columns up to 64 query rows, else 2 of 128) and their distance
     uint32_t tmem;
     unsigned char *kring, *vring, *qs, *ps;
@@ -318,6 +318,12 @@ __device__ __forceinline__ void cursor_next(Cursor& c, const AttnParams& p, cons
         cursor_open(c, p, cx, hi, lane);
     }
 }
+// Does the round at the cursor reach beyond the prefix?  (whole warp; tile ids ascend)
+__device__ __forceinline__ bool cursor_beyond_prefix(const Cursor& c, int P)
+{
+    const int nt = c.jn - c.k < 2 ? 1 : 2;
+    return __shfl_sync(0xffffffffu, c.my_tile, (c.k + nt - 1) & 31) * TILE + TILE > P;
+}
 // The round at the cursor: two tiles (rows 0-63 and 64-127 of both 64-column panels) into one stage.
 __device__ __forceinline__ void cursor_issue(const Cursor& c, const CUtensorMap* tm, unsigned char* ring, uint32_t full, uint64_t pol, int lane)
 {
@@ -351,11 +357,18 @@ __device__ __forceinline__ void producer_loop(const AttnParams& p, const Ctx& cx
     cv = ck;
     int ok = 1;
     uint32_t idle = 0;
+    int app_ok = p.app_row == nullptr;               // rows appended by this kernel are in place (tiles beyond the prefix may be loaded)
     while ((ck.live || cv.live) && ok) {
+        if (!app_ok) {
+            const int done = lane == 0 ? (int)mbar_try(cx.app_done, 0) : 0;
+            app_ok = __shfl_sync(0xffffffffu, done, 0);
+        }
+        const bool hold_k = !app_ok && ck.live && cursor_beyond_prefix(ck, p.P);
+        const bool hold_v = !app_ok && cv.live && cursor_beyond_prefix(cv, p.P);
         int rk = 0, rv = 0;
         if (lane == 0) {
-            rk = ck.live && mbar_try(cx.k_empty + 8 * ck.st, ck.ph ^ 1);
-            rv = cv.live && mbar_try(cx.v_empty + 8 * cv.st, cv.ph ^ 1);
+            rk = ck.live && !hold_k && mbar_try(cx.k_empty + 8 * ck.st, ck.ph ^ 1);
+            rv = cv.live && !hold_v && mbar_try(cx.v_empty + 8 * cv.st, cv.ph ^ 1);
         }
         rk = __shfl_sync(0xffffffffu, rk, 0);
         rv = __shfl_sync(0xffffffffu, rv, 0);
@@ -495,6 +508,63 @@ __device__ __noinline__ void clear_unseen_rows(uint32_t vs, const uint64_t* un, 
     __syncwarp();
 }
 
+// Fused append (one warp; out of line, all arguments by value).  The new K/V vectors of this pass
+// (Sec. 3.3: every emitted token's K/V is written once, at the row its slot reserves) whose rows
+// lie in KV tiles that this CTA owns are written here, before the CTA loads those tiles: every
+// tile of a (scene, KV head) pair belongs to exactly one CTA, so every vector is written exactly
+// once and no CTA depends on another.  Lanes 0-15 copy the 16 chunks of a K row, lanes 16-31
+// those of the V row.  Rows outside [P, rows) are skipped and flagged.  The writes are made
+// visible to the TMA loads (asynchronous proxy) of this CTA before the caller signals them.
+__device__ __noinline__ void append_rows(char* kc, char* vc, long long stride_scene_b, long long stride_head_b, long long stride_row_b,
+                                         const int32_t* app_row, const char* app_k, const char* app_v, const int32_t* tiles,
+                                         int ntile_max, int max_active, int hkv, int rows, int P, const int* pre, const int* nact,
+                                         long long lo, long long hi, int32_t* status)
+{
+    const int lane = threadIdx.x & 31;
+    const int chunk = (lane & 15) * 16;
+    const char* src_base = lane < 16 ? app_k : app_v;
+    char* dst_base = lane < 16 ? kc : vc;
+    int s = 0;
+    long long u = lo;
+    while (u < hi) {
+        const Segment sg = decode_segment(u, hi, pre, hkv, s);
+        const int A = nact[sg.s];
+        const int t_first = tiles[(size_t)sg.s * ntile_max + sg.j0], t_last = tiles[(size_t)sg.s * ntile_max + sg.j1 - 1];
+        for (int b0 = 0; b0 < A; b0 += 32) {
+            const int b = b0 + lane;
+            const int r = b < A ? app_row[(size_t)sg.s * max_active + b] : P;
+            const bool in_range = r >= P && r < rows;
+            if (!in_range && sg.g == 0 && sg.j0 == 0) atomicOr(status, FDC_DEV_ROW_RANGE);      // once per scene
+            const int t = r / TILE;
+            unsigned m = __ballot_sync(0xffffffffu, b < A && in_range && t >= t_first && t <= t_last);
+            while (m) {
+                // up to four rows per turn, all loads before the first store
+                uint4 val[4];
+                long long dst[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    dst[i] = -1;
+                    if (m) {
+                        const int bi = __ffs(m) - 1;
+                        m &= m - 1;
+                        const int ri = __shfl_sync(0xffffffffu, r, bi);
+                        const size_t slot = (size_t)sg.s * max_active + b0 + bi;
+                        val[i] = *reinterpret_cast<const uint4*>(src_base + (slot * hkv + sg.g) * (D * 2) + chunk);
+                        dst[i] = (long long)sg.s * stride_scene_b + (long long)sg.g * stride_head_b + (long long)ri * stride_row_b + chunk;
+                    }
+                }
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+                    if (dst[i] >= 0) *reinterpret_cast<uint4*>(dst_base + dst[i]) = val[i];
+            }
+        }
+        u = sg.next_u;
+    }
+    __threadfence();
+    asm volatile("fence.proxy.async;" ::: "memory");
+    __syncwarp();
+}
+
 // One warp: the V rows of a stage that are invisible to every branch of the scene are cleared
 // before the stage is multiplied.  Their P^T row is exactly 0, but the rows can hold anything
 // (NaN, Inf: slots that were never written) and 0 * NaN must not reach the accumulator.  Stages
@@ -502,6 +572,15 @@ __device__ __noinline__ void clear_unseen_rows(uint32_t vs, const uint64_t* un, 
 // runs ahead (as far as the V ring is deep) instead of delaying the multiplications.
 __device__ __forceinline__ void clean_loop(const AttnParams& p, const Ctx& cx, long long lo, long long hi, int lane)
 {
+    if (p.app_row) {
+        // a recorded fdc_kv_append: this warp writes the rows that fall into the CTA's tiles, then lets
+        // the producer go on to the tiles beyond the prefix
+        append_rows(const_cast<char*>(reinterpret_cast<const char*>(p.k)), const_cast<char*>(reinterpret_cast<const char*>(p.v)),
+                    p.stride_scene * 2, p.stride_head * 2, p.stride_row * 2, p.app_row, reinterpret_cast<const char*>(p.app_k),
+                    reinterpret_cast<const char*>(p.app_v), p.tiles, p.ntile_max, p.max_active, p.hkv, p.rows, p.P, cx.pre, cx.nact, lo, hi,
+                    p.status);
+        if (lane == 0) mbar_arrive(cx.app_done);
+    }
     int s = 0;
     uint32_t seg = 0;
     int st = 0;
@@ -1173,7 +1252,8 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, con
     cx.pv_done = cx.p_full + 16;
     cx.q_ready = cx.pv_done + 16;
     cx.o_free = cx.q_ready + 8;
-    uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bars + 5 * MAXST + 14);
+    cx.app_done = cx.o_free + 8;
+    uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bars + 5 * MAXST + 16);
     cx.mneg = reinterpret_cast<float*>(tmem_holder + 4);
     cx.alpha = cx.mneg + 128;
     cx.lred = cx.alpha + 128;
@@ -1211,6 +1291,7 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, con
         }
         mbar_init(cx.q_ready, NSOFT);
         mbar_init(cx.o_free, NSOFT);
+        mbar_init(cx.app_done, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         fence_async_smem();
     }
@@ -1464,7 +1545,7 @@ int launch_attn_tc(const AttnParams& p, int head_dim, cudaStream_t st)
     const int np_max = p.mmax <= 32 ? 32 : (p.mmax <= 64 ? 64 : 128);
     const int p_buf = ((np_max + 63) / 64) * PANEL;
     const int npb = np_max > 64 ? 1 : 2;          // 128 query rows: one P^T buffer, so that four stages still fit
-    const size_t fixed = 1024 + (size_t)npb * p_buf + (size_t)(D / 64) * np_max * 128 + 8 * (5 * MAXST + 14) + 16 +
+    const size_t fixed = 1024 + (size_t)npb * p_buf + (size_t)(D / 64) * np_max * 128 + 8 * (5 * MAXST + 16) + 16 +
                          4 * (128 + 128 + 512 + 128 + 8) + sizeof(int) * (3 * p.batch + 2) + 8 * (2 * MBUF + 2 * UW + 2) + 64;
     int stages = (int)((227 * 1024 - 256 - fixed) / STAGE);
     if (stages > 2 * MAXST) stages = 2 * MAXST;

@@ -46,6 +46,18 @@ struct alignas(16) SceneState {
 
 }  // namespace fdc
 
+// Arguments of an fdc_kv_append call that has been recorded instead of launched (fused append).
+struct fdc_pending_append {
+    int            valid;
+    fdc_kv_desc    kv;
+    int32_t        layer;
+    const int32_t* d_n_active;
+    const int32_t* d_kv_row;
+    const void*    d_k_new;
+    const void*    d_v_new;
+    void*          stream;
+};
+
 struct fdc_plan {
     fdc::PlanDev  h;                 // host copy
     fdc::PlanDev* d;                 // device copy
@@ -54,6 +66,8 @@ struct fdc_plan {
     int32_t*      d_pair_cnt;        // [FDC_PAIR_COUNTERS] arrivals per (scene, KV head) of the fused combine (zero between calls)
     int32_t*      d_split_memo;      // [2][FDC_MEMO_INTS] work split of the last attention launch and the counts it was made from
     uint32_t      attn_seq;          // attention launches on this plan so far (selects the memo slot)
+    int           fuse_append;       // fdc_set_fused_append
+    fdc_pending_append pend;         // recorded append waiting for its attention call
     int           device;
     int           sm_count;
     int           attn_kernel;       // 0 auto
@@ -84,6 +98,9 @@ struct AttnParams {
     int32_t*        pair_cnt;        // per (scene, KV head) arrival counters: the split kernel also combines (nullptr: it does not)
     int32_t*        split_memo;      // [2][FDC_MEMO_INTS] (nullptr: the work split is always computed)
     uint32_t        seq;             // number of this launch on the plan
+    const int32_t*  app_row;         // fused append: [batch][max_active] cache row of each branch's new K/V vector (nullptr: none)
+    const void*     app_k;           // [batch][max_active][hkv][D]
+    const void*     app_v;
 };
 
 extern int64_t g_launches;
@@ -96,6 +113,10 @@ int launch_attn_tc(const AttnParams& p, int head_dim, cudaStream_t st);
 int launch_attn_combine(const AttnParams& p, int dtype, int head_dim, cudaStream_t st);
 void prof_destroy(fdc_plan* plan);
 int  check_kv_desc(const fdc_plan* plan, const fdc_kv_desc* kv, int32_t layer);
+bool takes_tc_kernel(const fdc_plan* plan, const fdc_kv_desc* kv);   // fdc_decode_attn would run the tcgen05 kernel with the combine fused in
+int  launch_kv_append(const fdc_plan* plan, const fdc_kv_desc* kv, int32_t layer, const int32_t* d_n_active, const int32_t* d_kv_row,
+                      const void* d_k_new, const void* d_v_new, void* stream);
+int  flush_pending_append(const fdc_plan* plan);     // launches a recorded append on its own (no-op when there is none)
 
 // ----------------------------------------------------------------------------------
 // device helpers

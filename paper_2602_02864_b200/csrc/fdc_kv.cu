@@ -89,13 +89,11 @@ int check_kv_desc(const fdc_plan* p, const fdc_kv_desc* kv, int32_t layer)
 
 }  // namespace fdc
 
-extern "C" int fdc_kv_append(const fdc_plan* p, const fdc_kv_desc* kv, int32_t layer, const int32_t* d_n_active,
-                             const int32_t* d_kv_row, const void* d_k_new, const void* d_v_new, void* stream)
+namespace fdc {
+
+int launch_kv_append(const fdc_plan* p, const fdc_kv_desc* kv, int32_t layer, const int32_t* d_n_active, const int32_t* d_kv_row,
+                     const void* d_k_new, const void* d_v_new, void* stream)
 {
-    int rc = check_kv_desc(p, kv, layer);
-    if (rc) return rc;
-    if (!d_n_active || !d_kv_row || !d_k_new || !d_v_new) return FDC_ERR_NULL;
-    if (((uintptr_t)d_k_new & 15) || ((uintptr_t)d_v_new & 15)) return FDC_ERR_SHAPE;
     const int es = kv->dtype == FDC_F32 ? 4 : 2;
     char* kb = (char*)kv->k + (size_t)layer * kv->stride_layer * es;
     char* vb = (char*)kv->v + (size_t)layer * kv->stride_layer * es;
@@ -122,4 +120,40 @@ extern "C" int fdc_kv_append(const fdc_plan* p, const fdc_kv_desc* kv, int32_t l
     }
     note_launch();
     return FDC_OK;
+}
+
+int flush_pending_append(const fdc_plan* plan)
+{
+    fdc_plan* p = const_cast<fdc_plan*>(plan);
+    if (!p || !p->pend.valid) return FDC_OK;
+    p->pend.valid = 0;
+    return launch_kv_append(p, &p->pend.kv, p->pend.layer, p->pend.d_n_active, p->pend.d_kv_row, p->pend.d_k_new, p->pend.d_v_new,
+                            p->pend.stream);
+}
+
+}  // namespace fdc
+
+extern "C" int fdc_kv_append(const fdc_plan* p, const fdc_kv_desc* kv, int32_t layer, const int32_t* d_n_active,
+                             const int32_t* d_kv_row, const void* d_k_new, const void* d_v_new, void* stream)
+{
+    int rc = check_kv_desc(p, kv, layer);
+    if (rc) return rc;
+    if (!d_n_active || !d_kv_row || !d_k_new || !d_v_new) return FDC_ERR_NULL;
+    if (((uintptr_t)d_k_new & 15) || ((uintptr_t)d_v_new & 15)) return FDC_ERR_SHAPE;
+    rc = flush_pending_append(p);                 // an earlier recorded append never met its attention call
+    if (rc) return rc;
+    if (p->fuse_append && takes_tc_kernel(p, kv)) {
+        // recorded only: the next fdc_decode_attn for this cache, layer and stream writes the rows itself
+        fdc_pending_append& pe = const_cast<fdc_plan*>(p)->pend;
+        pe.kv = *kv;
+        pe.layer = layer;
+        pe.d_n_active = d_n_active;
+        pe.d_kv_row = d_kv_row;
+        pe.d_k_new = d_k_new;
+        pe.d_v_new = d_v_new;
+        pe.stream = stream;
+        pe.valid = 1;
+        return FDC_OK;
+    }
+    return launch_kv_append(p, kv, layer, d_n_active, d_kv_row, d_k_new, d_v_new, stream);
 }

@@ -234,6 +234,10 @@ int fdc_state_init(const fdc_plan* p, int32_t batch, const int32_t* d_len, void*
 {
     if (!p || !d_state) return FDC_ERR_NULL;
     if (batch < 1 || batch > FDC_MAX_BATCH) return FDC_ERR_RANGE;
+    {
+        int rcf = flush_pending_append(p);
+        if (rcf) return rcf;
+    }
     const int warps = 4;
     state_init_kernel<<<(batch + warps - 1) / warps, warps * 32, 0, (cudaStream_t)stream>>>(
         p->d, batch, d_len, (SceneState*)d_state, p->d_status);
@@ -249,6 +253,10 @@ int fdc_frontier(const fdc_plan* p, int32_t batch, void* d_state, const uint8_t*
     if (!p || !d_state || !d_n_active || !d_node || !d_tok_idx || !d_kv_row || !d_pos_id || !d_all_done)
         return FDC_ERR_NULL;
     if (batch < 1 || batch > FDC_MAX_BATCH) return FDC_ERR_RANGE;
+    {
+        int rcf = flush_pending_append(p);
+        if (rcf) return rcf;
+    }
     const int warps = batch < 8 ? batch : 8;
     frontier_kernel<<<(batch + warps - 1) / warps, warps * 32, 0, (cudaStream_t)stream>>>(
         p->d, batch, (SceneState*)d_state, d_finish, d_n_active, d_node, d_tok_idx, d_kv_row, d_pos_id,
@@ -263,6 +271,10 @@ int fdc_build_masks(const fdc_plan* p, int32_t batch, const void* d_state, uint6
 {
     if (!p || !d_state || !d_mask || !d_umask || !d_tiles || !d_ntiles) return FDC_ERR_NULL;
     if (batch < 1 || batch > FDC_MAX_BATCH) return FDC_ERR_RANGE;
+    {
+        int rcf = flush_pending_append(p);
+        if (rcf) return rcf;
+    }
     build_masks_kernel<<<batch, 256, p->h.W * sizeof(uint64_t), (cudaStream_t)stream>>>(
         p->d, (const SceneState*)d_state, d_mask, d_umask, d_tiles, d_ntiles);
     note_launch();

@@ -73,6 +73,7 @@ _decode_attn_static = _sig("fdc_decode_attn_static", c_i32, c_vp, ctypes.POINTER
                            c_vp, c_vp, c_vp, ctypes.c_float, c_vp)
 _status = _sig("fdc_status", c_i32, c_vp, ctypes.POINTER(c_i32), c_i32, c_vp)
 _set_attn_kernel = _sig("fdc_set_attn_kernel", c_i32, c_vp, c_i32)
+_set_fused_append = _sig("fdc_set_fused_append", c_i32, c_vp, c_i32)
 _kernel_name = _sig("fdc_kernel_name", ctypes.c_char_p, c_i32)
 _profile = _sig("fdc_profile", c_i32, c_vp, c_i32)
 _profile_read = _sig("fdc_profile_read", c_i32, c_vp, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_float),
@@ -214,6 +215,10 @@ def fdc_set_attn_kernel(plan, which: int) -> None:
     _check(_set_attn_kernel(plan, which), "fdc_set_attn_kernel")
 
 
+def fdc_set_fused_append(plan, on: bool) -> None:
+    _check(_set_fused_append(plan, 1 if on else 0), "fdc_set_fused_append")
+
+
 def fdc_kernel_name(which: int) -> Optional[str]:
     s = _kernel_name(which)
     return s.decode() if s else None
@@ -279,6 +284,7 @@ class DecodeSession:
         self.workspace = None
         self.ws_bytes = 0
         self.kv = None
+        self._append_refs = None
 
     def close(self):
         if self.plan:
@@ -313,10 +319,16 @@ class DecodeSession:
 
     def kv_append(self, layer, k_new, v_new, stream=None) -> None:
         fdc_kv_append(self.plan, self.kv, layer, self.n_active, self.kv_row, k_new, v_new, stream)
+        self._append_refs = (k_new, v_new)      # a recorded (fused) append reads them in the next decode_attn
 
     def decode_attn(self, layer, q, out, scale, stream=None) -> None:
         fdc_decode_attn(self.plan, self.kv, layer, self.n_active, self.mask, self.tiles, self.ntiles, q, out, scale,
                         self.workspace, self.ws_bytes, stream)
+        self._append_refs = None
+
+    def set_fused_append(self, on: bool) -> None:
+        """fdc_set_fused_append: kv_append is recorded and carried out by the next decode_attn."""
+        fdc_set_fused_append(self.plan, on)
 
     def status(self, clear=False) -> int:
         return fdc_status(self.plan, clear)

@@ -93,7 +93,8 @@ def check_close(got: np.ndarray, ref: np.ndarray, dtype: str, what=""):
 
 
 def run_and_compare(w: wl.Workload, check_steps=None, check_layers=None, extra_rows: int = 0,
-                    use_finish_flags: bool = False, kernel: int = 0, device="cuda", max_steps=None):
+                    use_finish_flags: bool = False, kernel: int = 0, device="cuda", max_steps=None,
+                    fused_append: bool = False):
     """Plays the whole schedule on the GPU through the C ABI and on the CPU checker.
     Integers are compared at every pass; attention at `check_steps` x `check_layers`
     (None = all).  Returns summary statistics."""
@@ -102,6 +103,8 @@ def run_and_compare(w: wl.Workload, check_steps=None, check_layers=None, extra_r
     sess = fdc.DecodeSession(w.n_nodes, w.edges, w.slot_cap, w.n_fixed, w.prefix_len, w.max_active, w.batch, device)
     if kernel:
         fdc.fdc_set_attn_kernel(sess.plan, kernel)
+    if fused_append:          # appends are recorded and written by the attention kernel (or on their own when none follows)
+        sess.set_fused_append(True)
     k, v = alloc_cache(w, device, extra_rows)
     write_prefix(w, k, v, oracle)
     sess.bind_cache(k, v, w.hq)

@@ -22,9 +22,10 @@ def _built():
     build.build()
 
 
-def _run(name, n_steps, samples):
+def _run(name, n_steps, samples, fused_append=True):
     """samples: list of (step, layer, scene)."""
     bench.LAYERS_OVERRIDE = None
+    bench.FUSED_APPEND = fused_append
     w = bench.get_workload(name)
     sb = bench.StepBench(w, n_steps, torch.device("cuda", 0))
     sb.reset()
@@ -64,9 +65,10 @@ def _run(name, n_steps, samples):
     return checked
 
 
-def test_cfg2_batched_full_size_sampled():
+@pytest.mark.parametrize("fused_append", [True, False], ids=["append_inside_attention", "append_kernel"])
+def test_cfg2_batched_full_size_sampled(fused_append):
     # 16 scenes x 32 layers x 8 KV heads x (4096 + 768) rows: the benchmark's headline workload
-    n = _run("cfg2", 24, [(0, 0, 0), (5, 31, 15), (17, 13, 7), (23, 20, 3), (23, 0, 9)])
+    n = _run("cfg2", 24, [(0, 0, 0), (5, 31, 15), (17, 13, 7), (23, 20, 3), (23, 0, 9)], fused_append)
     assert n > 0
 
 

@@ -237,3 +237,77 @@ def test_work_split_of_the_previous_call_is_reused_only_for_the_same_counts():
     assert torch.equal(first, back)
     assert sess.status() == 0
     sess.close()
+
+
+@pytest.mark.parametrize("which", ["cfg1", "cfg2", "cfg3", "ragged", "fixed_rows"])
+def test_fused_append_writes_the_same_cache_and_gives_the_same_attention(which):
+    """fdc_set_fused_append: kv_append is only recorded and the next decode_attn writes the rows
+    inside its kernel.  The whole schedule is played with the option on; layers / passes whose
+    attention is not checked have no matching attention call, so their appends take the
+    stand-alone kernel when the next call flushes them.  Attention matches the checker and at
+    the end the whole cache equals the checker's, bit for bit (every real row once, padding never)."""
+    if which == "cfg1":
+        w = wl.cfg1_7b(layers=2)
+        r = run_and_compare(w, check_steps=set(range(0, 200, 7)), check_layers={1}, fused_append=True)
+    elif which == "cfg2":
+        w = wl.cfg2_batched(layers=1, batch=4)
+        r = run_and_compare(w, check_steps=set(range(0, 300, 5)) | {15, 16, 95, 96}, fused_append=True)
+    elif which == "cfg3":
+        w = wl.cfg3_wide(layers=1, batch=2)
+        r = run_and_compare(w, check_steps=set(range(0, 144, 3)), fused_append=True)
+    elif which == "ragged":      # prefix length that is no tile multiple, cache longer than P + T, bf16 head_dim 128
+        w = wl.random_template(3006, n_nodes=9, edge_prob=0.3, cap_lo=2, cap_hi=70, batch=3, prefix_len=200, fixed_hi=0,
+                               hq=8, hkv=2, head_dim=128, dtype="bf16")
+        w.max_active = w.n_nodes
+        r = run_and_compare(w, extra_rows=30, fused_append=True)
+    else:                         # fixed field-name rows ahead of the generated tokens, prefix of 0 rows
+        w = wl.random_template(3000, n_nodes=5, edge_prob=0.3, cap_lo=2, cap_hi=70, batch=3, prefix_len=0, fixed_hi=3,
+                               hq=8, hkv=2, head_dim=128, dtype="bf16")
+        w.max_active = w.n_nodes
+        r = run_and_compare(w, fused_append=True)
+    assert r["checked"] > 0
+
+
+def test_fused_append_is_carried_out_even_without_an_attention_call():
+    """A recorded append must never be lost: fdc_status, a second append, an attention call for
+    another layer and switching the option off each launch it on its own first."""
+    from paper_2602_02864_b200 import fdc
+    from harness import alloc_cache, write_prefix
+    w = wl.cfg2_batched(layers=2, batch=2)
+    dev = "cuda"
+    sess = fdc.DecodeSession(w.n_nodes, w.edges, w.slot_cap, w.n_fixed, w.prefix_len, w.max_active, w.batch, dev)
+    k, v = alloc_cache(w, dev, fill=0.0)
+    write_prefix(w, k, v)
+    sess.bind_cache(k, v, w.hq)
+    sess.init(torch.from_numpy(w.lens).to(dev))
+    sess.set_fused_append(True)
+    sess.frontier(None)
+    sess.build_masks()
+    rows = sess.kv_row.cpu().numpy()
+    n_act = sess.n_active.cpu().numpy()
+
+    def written(layer, kn):
+        torch.cuda.synchronize()
+        for s in range(w.batch):
+            for b in range(int(n_act[s])):
+                if not torch.equal(k[s, layer, :, int(rows[s, b])], kn[s, b]):
+                    return False
+        return True
+
+    launches = fdc.fdc_launch_count()
+    q, kn0, vn0 = wl.step_qkv(w, 0, 0, dev)
+    sess.kv_append(0, kn0, vn0)
+    assert fdc.fdc_launch_count() == launches            # recorded, nothing launched
+    assert sess.status() == 0                            # fdc_status flushes
+    assert written(0, kn0)
+    _, kn1, vn1 = wl.step_qkv(w, 0, 1, dev)
+    sess.kv_append(1, kn1, vn1)
+    out = torch.zeros_like(q)
+    sess.decode_attn(0, q, out, w.softmax_scale)         # attention for ANOTHER layer: append of layer 1 goes first, on its own
+    assert written(1, kn1)
+    _, kn2, vn2 = wl.step_qkv(w, 1, 0, dev)
+    sess.kv_append(0, kn2, vn2)
+    sess.set_fused_append(False)                         # switching off flushes too
+    assert written(0, kn2)
+    assert sess.status() == 0
+    sess.close()
