@@ -10,20 +10,26 @@
 //                      as TMA left them in shared memory, B = Q^T staged once per segment
 //     O^T += V^T P^T   M = head_dim, N = NP, K = 128 KV rows;  A = the V tiles (M-major), B =
 //                      P^T written by the softmax threads (N-major), accumulator in TMEM
-// One persistent CTA per SM:
-//   warps 16, 18 TMA producers: K stages and V stages (128 rows, 128B swizzle) of two rings
-//   warp 17      issues S^T = K Q^T (one elected thread); allocates / frees TMEM.  S^T is double
-//                buffered in TMEM, so K Q^T of round r+1 overlaps the softmax of round r
-//   warp 19      clears the V rows that no branch may see (they can hold anything, NaN included,
-//                and 0 * NaN must not reach the accumulator), then issues O^T += V^T P^T
+// One persistent CTA per SM, 20 warps:
+//   warp 16      TMA producer of both rings (K stages and V stages: 128 rows, 128B swizzle, L2
+//                evict-first); polls both rings' free barriers, never blocks on one of them
+//   warp 17      issues S^T = K Q^T (one elected thread); allocates / frees TMEM.  S^T has four
+//                buffers in TMEM (two for 128 query rows), so K Q^T runs ahead of the softmax
+//   warp 18      with fdc_set_fused_append, first writes the pass's new K/V rows that fall into
+//                this CTA's tiles; then clears, ahead of the multiplications, the V rows that no
+//                branch may see (they can hold anything, NaN included, and 0 * NaN must not reach
+//                the accumulator) and passes each V stage on
+//   warp 19      issues O^T += V^T P^T (one elected thread)
 //   warps 0-15   softmax.  Thread = one KV row of the round (TMEM lane) x a quarter of the query
 //                columns.  Eq. 1 is applied by select from the branches' row bitmaps; prefix
 //                tiles skip it.
-// The softmax reference of a query column is raised lazily: it is set from the column maximum
-// of the first round (a column that sees no row yet borrows the round's highest maximum).  A
-// score more than 2^16 above its reference leaves a note that all warps act on two rounds later
-// (no barrier in the common path); a rise of more than 2^100 within those two rounds is flagged.  Sum and accumulator use the same reference, so the
-// result is exact; the column sums are kept per thread and reduced at the end of a segment.
+// The softmax reference of a query column is set in the first round of a segment: inside the
+// prefix from the score against the round's first row (visible to everybody), else from the
+// column maximum (a column that sees no row yet borrows the round's highest maximum).  A score
+// more than 2^16 above its reference leaves a note that all warps act on two rounds later (no
+// barrier in the common path); a rise of more than 2^100 within those two rounds is flagged.
+// Sum and accumulator use the same reference, so the result is exact; the column sums are kept
+// per thread in TMEM and reduced at the end of a segment.
 #include <cudaTypedefs.h>
 
 #include <climits>
@@ -41,7 +47,7 @@ constexpr int NSOFT = 16;                    // softmax warps: 4 row quadrants x
 constexpr int NPART = NSOFT / 4;             // column parts
 constexpr int W_PROD = NSOFT, W_QK = NSOFT + 1, W_CLEAN = NSOFT + 2, W_PV = NSOFT + 3;
 constexpr int THREADS = (NSOFT + 4) * 32;
-constexpr uint32_t TMEM_COLS = 512;          // S^T 0 [0,128) | S^T 1 [128,256) | O^T [256,384) | sums [384,512)
+constexpr uint32_t TMEM_COLS = 512;          // S^T buffers [0,256): 4 x 64 columns (2 x 128 for 128 query rows) | O^T [256,384) | sums [384,512)
 constexpr uint32_t TM_O = 256;
 constexpr uint32_t TM_L = 384;                // per-column sums of the softmax threads [384, 512)
 constexpr int PANEL = RROWS * 128;           // 128 rows x 128 bytes (64 bf16 columns)
@@ -83,16 +89,8 @@ __device__ __forceinline__ uint32_t instr_desc(int m, int n, uint32_t mn_major)
     return (1u << 4) | (1u << 7) | (1u << 10) | (mn_major << 15) | (mn_major << 16) | ((uint32_t)(n >> 3) << 17) |
            ((uint32_t)(m >> 4) << 24);
 }
-__device__ __forceinline__ void umma(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate)
-{
-    asm volatile(
-        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
-        : "memory");
-}
-// The same with the descriptors given as (low, high) words: the address field sits in the low
-// word, so stepping through an operand is 32-bit arithmetic for the issuing thread.
+// One MMA (cta_group::1, kind::f16).  The descriptors are given as (low, high) words: the address
+// field sits in the low word, so stepping through an operand is 32-bit arithmetic for the issuing thread.
 __device__ __forceinline__ void umma2(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi, uint32_t idesc,
                                       uint32_t accumulate)
 {
@@ -151,16 +149,6 @@ __device__ __forceinline__ void tmem_st(uint32_t taddr, const uint32_t (&v)[N])
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
-// OR of a predicate over the softmax threads (named barrier 1)
-__device__ __forceinline__ bool soft_any(bool x)
-{
-    uint32_t out;
-    asm volatile("{\n\t.reg .pred p, q;\n\tsetp.ne.u32 q, %1, 0;\n\tbar.red.or.pred p, 1, %2, q;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-                 : "=r"(out)
-                 : "r"((uint32_t)x), "n"(NSOFT * 32)
-                 : "memory");
-    return out != 0;
-}
 __device__ __forceinline__ void soft_sync() { asm volatile("bar.sync 1, %0;" ::"n"(NSOFT * 32) : "memory"); }
 
 __device__ __forceinline__ uint32_t pack2(float lo, float hi)
@@ -196,11 +184,6 @@ struct Ctx {
     long long vtot;                  // total weighted length
     volatile int* abortp;
     int nk, nv, q_panel, p_buf, npb; // ring depths, bytes per 64-column panel of Q^T, bytes per P^T buffer, P^T buffers (1 or 2)
-};
-
-// A round: up to two entries of a segment's tile list.
-struct Round {
-    int nt, tile0, tile1;
 };
 
 // Row bitmap (Eq. 1) of branch b of the segment's scene.  While the K/V stream saturates the
