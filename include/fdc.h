@@ -71,9 +71,12 @@ enum {
     FDC_DEV_LEN_RANGE     = 4,  /* fdc_state_init: a length outside [n_fixed+1, C]: clamped  */
     FDC_DEV_TIMEOUT       = 8,  /* fdc_decode_attn: a bounded in-kernel wait ran out; the    */
                                 /* launch's output is invalid                                */
-    FDC_DEV_SCORE_RANGE   = 16  /* fdc_decode_attn: a score rose more than 2^100 above its   */
+    FDC_DEV_SCORE_RANGE   = 16, /* fdc_decode_attn: a score rose more than 2^100 above its   */
                                 /* softmax reference within two rounds (128 KV rows each)    */
                                 /* of a reference update: the output may have overflowed     */
+    FDC_DEV_TILE_LIST     = 32  /* fdc_decode_attn: d_tiles does not list the whole prefix   */
+                                /* tiles first, as entries 0, 1, 2, ... (fdc_build_masks     */
+                                /* always does); rows nobody may see could have been read    */
 };
 
 typedef struct fdc_plan fdc_plan;
@@ -191,7 +194,9 @@ int fdc_attn_workspace_bytes(const fdc_plan* plan, const fdc_kv_desc* kv, size_t
  * [head_dim] in the cache dtype; rows of unused branch slots are not touched.  Scores,
  * softmax and accumulation are fp32; bf16 output is rounded to nearest even.  Each visited
  * KV tile is read once for all branches and all heads of its KV group; invisible K/V rows
- * may hold anything (NaN included).  d_workspace: DEVICE, 256-byte aligned,
+ * may hold anything (NaN included).  d_tiles must be what fdc_build_masks wrote: ascending,
+ * with entry j = tile j for every whole tile of the prefix (FDC_DEV_TILE_LIST otherwise).
+ * d_workspace: DEVICE, 256-byte aligned,
  * >= fdc_attn_workspace_bytes; its contents are undefined afterwards.
  * The tcgen05 kernel merges its split partials itself and keeps per-(scene, KV head) arrival
  * counters in the plan, and it leaves its work split there for the next call (checked against

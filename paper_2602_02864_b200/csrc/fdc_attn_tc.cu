@@ -183,6 +183,7 @@ struct Ctx {
     int npre;                        // tiles wholly inside the prefix
     long long vtot;                  // total weighted length
     volatile int* abortp;
+    volatile int* v_issued;          // V rounds the producer has requested so far (read by the cleaning warp)
     int nk, nv, q_panel, p_buf, npb; // ring depths, bytes per 64-column panel of Q^T, bytes per P^T buffer, P^T buffers (1 or 2)
 };
 
@@ -361,6 +362,7 @@ __device__ __forceinline__ void producer_loop(const AttnParams& p, const Ctx& cx
         }
         if (rv) {
             cursor_issue(cv, tm_v, cx.vring, cx.v_full, pol, lane);
+            if (lane == 0) *cx.v_issued = (int)cv.g + 1;
             cursor_next(cv, p, cx, hi, cx.nv, lane);
         }
         if (rk | rv) {
@@ -548,6 +550,19 @@ __device__ __noinline__ void append_rows(char* kc, char* vc, long long stride_sc
     __syncwarp();
 }
 
+// Bounded wait until the producer has requested V round g (*issued > g).
+__device__ __noinline__ int wait_issued(volatile int* issued, int g, volatile int* abort_flag, int32_t* status)
+{
+    for (uint32_t i = 0; i < SPIN_LIMIT; ++i) {
+        if (*issued > g) return 1;
+        if (*abort_flag) return 0;
+        __nanosleep(64);
+    }
+    *abort_flag = 1;
+    atomicOr(status, FDC_DEV_TIMEOUT);
+    return 0;
+}
+
 // One warp: the V rows of a stage that are invisible to every branch of the scene are cleared
 // before the stage is multiplied.  Their P^T row is exactly 0, but the rows can hold anything
 // (NaN, Inf: slots that were never written) and 0 * NaN must not reach the accumulator.  Stages
@@ -565,7 +580,7 @@ __device__ __forceinline__ void clean_loop(const AttnParams& p, const Ctx& cx, l
         if (lane == 0) mbar_arrive(cx.app_done);
     }
     int s = 0;
-    uint32_t seg = 0;
+    uint32_t seg = 0, g = 0;
     int st = 0;
     uint32_t vph = 0;
     long long u = lo;
@@ -577,23 +592,34 @@ __device__ __forceinline__ void clean_loop(const AttnParams& p, const Ctx& cx, l
         for (int jb = sg.j0; jb < sg.j1 && ok; jb += 32) {
             const int jn = sg.j1 - jb < 32 ? sg.j1 - jb : 32;
             const int my_tile = lane < jn ? p.tiles[(size_t)sg.s * p.ntile_max + jb + lane] : 0;
-            for (int k = 0; k < jn && ok; k += 2) {
+            for (int k = 0; k < jn && ok; k += 2, ++g) {
                 const int nt = jn - k < 2 ? 1 : 2;
                 // tile ids ascend: the round reaches beyond the prefix iff its last tile does
                 const int t_last = __shfl_sync(0xffffffffu, my_tile, (k + nt - 1) & 31);
                 const bool masked = t_last * TILE + TILE > p.P;
-                int okw = 1;
-                if (lane == 0) {
-                    okw = mbar_wait(cx.v_full + 8 * st, vph, cx.abortp, p.status);
-                    if (okw && masked && !have_masks) okw = mbar_wait(cx.q_ready, seg & 1, cx.abortp, p.status);
+                // Which rounds pass through this warp is decided by POSITION on both sides (entry j of a list
+                // is tile j inside the prefix), so the two can never disagree about the barrier; a list that
+                // breaks the rule is flagged (an uncleaned stage could have been multiplied).
+                const bool beyond = jb + k + nt - 1 >= p.P / TILE;
+                if (lane == 0 && masked != beyond) atomicOr(p.status, FDC_DEV_TILE_LIST);
+                if (beyond) {
+                    int okw = 1;
+                    if (lane == 0) {
+                        // Rounds inside the prefix are skipped without a wait, so this warp can be far ahead of
+                        // the ring: it first waits until the producer has requested round g (then the stage's
+                        // barrier cannot be in an earlier phase with the same parity), then for the data.
+                        okw = wait_issued(cx.v_issued, (int)g, cx.abortp, p.status);
+                        if (okw) okw = mbar_wait(cx.v_full + 8 * st, vph, cx.abortp, p.status);
+                        if (okw && masked && !have_masks) okw = mbar_wait(cx.q_ready, seg & 1, cx.abortp, p.status);
+                    }
+                    ok = __shfl_sync(0xffffffffu, okw, 0);
+                    if (ok && masked) {
+                        have_masks = true;
+                        clear_unseen_rows(smem_u32(cx.vring) + st * STAGE, (cx.mstaged && p.W <= UW) ? cx.sunion + (seg & 1) * UW : nullptr,
+                                          mask_row(p, cx, seg, sg.s, 0), p.W, p.P, A, __shfl_sync(0xffffffffu, my_tile, k & 31), t_last, nt);
+                    }
+                    if (ok && lane == 0) mbar_arrive(cx.v_clean + 8 * st);
                 }
-                ok = __shfl_sync(0xffffffffu, okw, 0);
-                if (ok && masked) {
-                    have_masks = true;
-                    clear_unseen_rows(smem_u32(cx.vring) + st * STAGE, (cx.mstaged && p.W <= UW) ? cx.sunion + (seg & 1) * UW : nullptr,
-                                      mask_row(p, cx, seg, sg.s, 0), p.W, p.P, A, __shfl_sync(0xffffffffu, my_tile, k & 31), t_last, nt);
-                }
-                if (ok && lane == 0) mbar_arrive(cx.v_clean + 8 * st);
                 if (++st == cx.nv) {
                     st = 0;
                     vph ^= 1;
@@ -613,10 +639,11 @@ __device__ __forceinline__ void pv_loop(const AttnParams& p, const Ctx& cx, long
     const uint64_t p_desc0 = smem_desc(smem_u32(cx.ps), PANEL, 1024);
     const uint32_t v_lo0 = (uint32_t)v_desc0, v_hi = (uint32_t)(v_desc0 >> 32), p_lo0 = (uint32_t)p_desc0, p_hi = (uint32_t)(p_desc0 >> 32);
     const uint32_t tm_o = cx.tmem + TM_O;
+    const int npre_tiles = p.P / TILE;
     int s = 0;
     uint32_t g = 0, seg = 0;
     int st = 0;
-    uint32_t vph = 0;
+    uint32_t vph = 0, cpar = 0;
     long long u = lo;
     int ok = 1;
     while (u < hi && ok) {
@@ -629,7 +656,17 @@ __device__ __forceinline__ void pv_loop(const AttnParams& p, const Ctx& cx, long
             bool good = true;
             for (int t = 0; 2 * t < ntile && good; ++t, ++g) {
                 const int nt = ntile - 2 * t < 2 ? 1 : 2;
-                good = mbar_wait(cx.v_clean + 8 * st, vph, cx.abortp, p.status);
+                // Entry j of a tile list is tile j for every whole prefix tile, so the position tells whether
+                // the round reaches beyond the prefix.  Only then does the stage come through the cleaning
+                // warp (which may still be busy with the append at the start of the CTA); v_clean[st]
+                // completes one phase per such round, counted in cpar on both sides.
+                const bool beyond = sg.j0 + 2 * t + nt - 1 >= npre_tiles;
+                if (beyond) {
+                    good = mbar_wait(cx.v_clean + 8 * st, (cpar >> st) & 1u, cx.abortp, p.status);
+                    cpar ^= 1u << st;
+                } else {
+                    good = mbar_wait(cx.v_full + 8 * st, vph, cx.abortp, p.status);
+                }
                 if (good) good = mbar_wait(cx.p_full + 8 * (g & 1), (g >> 1) & 1, cx.abortp, p.status);
                 if (good && t == 0 && seg > 0) good = mbar_wait(cx.o_free, (seg - 1) & 1, cx.abortp, p.status);
                 if (!good) break;
@@ -655,6 +692,7 @@ __device__ __forceinline__ void pv_loop(const AttnParams& p, const Ctx& cx, long
         g = __shfl_sync(0xffffffffu, g, 0);
         st = __shfl_sync(0xffffffffu, st, 0);
         vph = __shfl_sync(0xffffffffu, vph, 0);
+        cpar = __shfl_sync(0xffffffffu, cpar, 0);
         ++seg;
         u = sg.next_u;
     }
@@ -1249,11 +1287,15 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, con
     cx.smask = reinterpret_cast<uint64_t*>(((uintptr_t)(cx.prev + p.batch + 1) + 7) & ~(uintptr_t)7);
     cx.sunion = cx.smask + 2 * MBUF;
     cx.mstaged = p.max_active * p.W <= MBUF;
-    __shared__ int abort_flag;
+    __shared__ int abort_flag, v_issued_count;
     cx.abortp = &abort_flag;
+    cx.v_issued = &v_issued_count;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    if (threadIdx.x == 0) abort_flag = 0;
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        v_issued_count = 0;
+    }
     if (threadIdx.x < 4) cx.rflag[threadIdx.x] = -1;
     // ---- set-up that needs no global memory: barriers, TMEM
     if (threadIdx.x == 0) {

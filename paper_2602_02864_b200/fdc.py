@@ -29,6 +29,7 @@ FDC_STATIC_WS_BYTES = 16 << 20
 FDC_F32, FDC_BF16 = 0, 1
 FDC_DEV_ROW_RANGE, FDC_DEV_FRONTIER_WIDE, FDC_DEV_LEN_RANGE, FDC_DEV_TIMEOUT = 1, 2, 4, 8
 FDC_DEV_SCORE_RANGE = 16
+FDC_DEV_TILE_LIST = 32
 
 c_i32, c_i64, c_vp, c_sz = ctypes.c_int32, ctypes.c_int64, ctypes.c_void_p, ctypes.c_size_t
 
