@@ -195,7 +195,8 @@ int fdc_attn_workspace_bytes(const fdc_plan* plan, const fdc_kv_desc* kv, size_t
  * softmax and accumulation are fp32; bf16 output is rounded to nearest even.  Each visited
  * KV tile is read once for all branches and all heads of its KV group; invisible K/V rows
  * may hold anything (NaN included).  d_tiles must be what fdc_build_masks wrote: ascending,
- * with entry j = tile j for every whole tile of the prefix (FDC_DEV_TILE_LIST otherwise).
+ * the whole tiles of the prefix first (entry j = tile j); the kernel decides by list position
+ * which tiles can hold rows that nobody may see (FDC_DEV_TILE_LIST if the list disagrees).
  * d_workspace: DEVICE, 256-byte aligned,
  * >= fdc_attn_workspace_bytes; its contents are undefined afterwards.
  * The tcgen05 kernel merges its split partials itself and keeps per-(scene, KV head) arrival

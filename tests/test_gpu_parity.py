@@ -311,3 +311,38 @@ def test_fused_append_is_carried_out_even_without_an_attention_call():
     assert written(0, kn2)
     assert sess.status() == 0
     sess.close()
+
+
+def test_tile_list_that_breaks_the_prefix_rule_is_flagged():
+    """The attention kernel decides by list position which V stages have to be cleaned of rows
+    nobody may see: the whole prefix tiles come first in a list (that is how fdc_build_masks
+    writes it).  A list with a tile from beyond the prefix among the prefix entries is reported
+    (the scene's output is then not to be trusted); the other scene is untouched and nothing
+    waits for ever."""
+    from paper_2602_02864_b200 import fdc
+    from harness import alloc_cache, write_prefix
+    w = wl.cfg2_batched(layers=1, batch=2)
+    dev = "cuda"
+    sess = fdc.DecodeSession(w.n_nodes, w.edges, w.slot_cap, w.n_fixed, w.prefix_len, w.max_active, w.batch, dev)
+    k, v = alloc_cache(w, dev, fill=0.0)
+    write_prefix(w, k, v)
+    sess.bind_cache(k, v, w.hq)
+    sess.init(torch.from_numpy(w.lens).to(dev))
+    sess.frontier(None)
+    sess.build_masks()
+    q, kn, vn = wl.step_qkv(w, 0, 0, dev)
+    sess.kv_append(0, kn, vn)
+    good = torch.zeros_like(q)
+    sess.decode_attn(0, q, good, w.softmax_scale)
+    assert sess.status() == 0
+    npre = w.prefix_len // 64
+    assert int(sess.ntiles[1]) > npre
+    tiles = sess.tiles.clone()
+    tiles[1, 3], tiles[1, npre] = sess.tiles[1, npre].clone(), sess.tiles[1, 3].clone()
+    out = torch.zeros_like(q)
+    fdc.fdc_decode_attn(sess.plan, sess.kv, 0, sess.n_active, sess.mask, tiles, sess.ntiles, q, out, w.softmax_scale,
+                        sess.workspace, sess.ws_bytes)
+    assert sess.status(clear=True) == fdc.FDC_DEV_TILE_LIST
+    assert torch.equal(out[0], good[0])
+    assert sess.status() == 0
+    sess.close()
