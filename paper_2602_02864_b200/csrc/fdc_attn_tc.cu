@@ -750,69 +750,59 @@ __device__ __noinline__ void prefetch_next_segment(const uint4* qg, const uint64
 }
 
 // Merge of the partials of one (scene, KV head) pair by the CTA that delivered the last one
-// (all softmax threads).  One thread per query row computes m = max_c m_c, l = sum_c l_c 2^(m_c - m)
-// and replaces m_c in the workspace by the weight 2^(m_c - m) / l; then every thread sums weighted
-// accumulator chunks.  Loads are issued four at a time: each costs a trip to L2 and none depends on
-// the previous one.  Out of line, arguments by value.
-__device__ __noinline__ void merge_pair(float* ws_ml, const float* ws_o, __nv_bfloat16* out, int pair, int mmax, int M, int G, int s, int g,
+// (all softmax threads).  Every thread owns four accumulator columns of one query row and merges
+// the parts' (m, l, O) for them in ONE pass, three parts per turn with all loads ahead of the
+// arithmetic (a turn costs one trip to L2; the running maximum is carried like in the online
+// softmax, so more parts need no second pass):
+//     m = max_c m_c,  l = sum_c l_c 2^(m_c - m),  O = sum_c O_c 2^(m_c - m) / l.
+// Out of line, arguments by value.
+__device__ __noinline__ void merge_pair(const float* ws_ml, const float* ws_o, __nv_bfloat16* out, int pair, int mmax, int M, int G, int s, int g,
                                         int max_active, int hq, int c_first, int c_last)
 {
+    constexpr int MB = 3;                          // parts per turn
     const int tid = threadIdx.x;
     __threadfence();
-    if (tid < M) {
-        float* ml = ws_ml + ((size_t)pair * mmax + tid) * 2;
-        const size_t cs = (size_t)mmax * 2;                // stride between CTAs' entries
-        float mx = -INFINITY;
-        for (int c0 = c_first; c0 <= c_last; c0 += 4) {
-            float v[4];
-#pragma unroll
-            for (int j = 0; j < 4; ++j) v[j] = c0 + j <= c_last ? __ldcg(ml + (size_t)(c0 + j) * cs) : -INFINITY;
-            mx = fmaxf(fmaxf(mx, fmaxf(v[0], v[1])), fmaxf(v[2], v[3]));
-        }
-        float lt = 0.f;
-        for (int c0 = c_first; c0 <= c_last; c0 += 4) {
-            float2 v[4];
-#pragma unroll
-            for (int j = 0; j < 4; ++j)
-                v[j] = c0 + j <= c_last ? __ldcg(reinterpret_cast<const float2*>(ml + (size_t)(c0 + j) * cs)) : make_float2(-INFINITY, 0.f);
-#pragma unroll
-            for (int j = 0; j < 4; ++j) lt = fmaf(v[j].y, fast_exp2(v[j].x - mx), lt);   // a split that saw nothing: -inf -> 0
-        }
-        const float inv = 1.f / lt;
-        for (int c = c_first; c <= c_last; ++c) {
-            const float w = fast_exp2(__ldcg(ml + (size_t)c * cs) - mx) * inv;
-            __stcg(ml + (size_t)c * cs, w);
-        }
-    }
-    __threadfence();
-    soft_sync();
     for (int idx = tid; idx < M * (D / 4); idx += NSOFT * 32) {
         const int m = idx / (D / 4), c4 = idx - m * (D / 4);
-        const float* ml = ws_ml + ((size_t)pair * mmax + m) * 2;
+        const float2* ml = reinterpret_cast<const float2*>(ws_ml + ((size_t)pair * mmax + m) * 2);
         const float4* po = reinterpret_cast<const float4*>(ws_o + ((size_t)pair * mmax + m) * D) + c4;
-        const size_t cs = (size_t)mmax * 2, os = (size_t)mmax * (D / 4);
+        const size_t cs = (size_t)mmax, os = (size_t)mmax * (D / 4);      // strides between CTAs' entries
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-        for (int c0 = c_first; c0 <= c_last; c0 += 4) {
-            float w[4];
-            float4 o[4];
+        float mx = -INFINITY, lt = 0.f;
+        for (int c0 = c_first; c0 <= c_last; c0 += MB) {
+            float2 v[MB];
+            float4 o[MB];
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
+            for (int j = 0; j < MB; ++j) {
                 const bool on = c0 + j <= c_last;
-                w[j] = on ? __ldcg(ml + (size_t)(c0 + j) * cs) : 0.f;
+                v[j] = on ? __ldcg(ml + (size_t)(c0 + j) * cs) : make_float2(-INFINITY, 0.f);
                 o[j] = on ? __ldcg(po + (size_t)(c0 + j) * os) : make_float4(0.f, 0.f, 0.f, 0.f);
             }
+            float nm = mx;
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                acc.x = fmaf(o[j].x, w[j], acc.x);
-                acc.y = fmaf(o[j].y, w[j], acc.y);
-                acc.z = fmaf(o[j].z, w[j], acc.z);
-                acc.w = fmaf(o[j].w, w[j], acc.w);
+            for (int j = 0; j < MB; ++j) nm = fmaxf(nm, v[j].x);
+            const float sc = mx == nm ? 1.f : fast_exp2(mx - nm);           // (-inf) - (-inf) must not be formed
+            lt *= sc;
+            acc.x *= sc;
+            acc.y *= sc;
+            acc.z *= sc;
+            acc.w *= sc;
+#pragma unroll
+            for (int j = 0; j < MB; ++j) {
+                const float w = v[j].x == -INFINITY ? 0.f : fast_exp2(v[j].x - nm);   // a part that saw nothing
+                lt = fmaf(v[j].y, w, lt);
+                acc.x = fmaf(o[j].x, w, acc.x);
+                acc.y = fmaf(o[j].y, w, acc.y);
+                acc.z = fmaf(o[j].z, w, acc.z);
+                acc.w = fmaf(o[j].w, w, acc.w);
             }
+            mx = nm;
         }
+        const float inv = 1.f / lt;
         const int b = m / G, hg = m - b * G;
         uint2 pk;
-        pk.x = pack2(acc.x, acc.y);
-        pk.y = pack2(acc.z, acc.w);
+        pk.x = pack2(acc.x * inv, acc.y * inv);
+        pk.y = pack2(acc.z * inv, acc.w * inv);
         *reinterpret_cast<uint2*>(out + (((size_t)s * max_active + b) * hq + (size_t)g * G + hg) * D + c4 * 4) = pk;
     }
 }
