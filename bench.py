@@ -214,8 +214,9 @@ class StepBench:
     def reset(self):
         self.sess.init(self.lens)
 
-    def step(self, i: int, q=None, kn=None, vn=None, log_masks: bool = False):
+    def step(self, i: int, q=None, kn=None, vn=None, log_masks: bool = False, out=None):
         s, w = self.sess, self.w
+        out = self.out if out is None else out
         q = self.q[i] if q is None else q
         kn = self.kn[i] if kn is None else kn
         vn = self.vn[i] if vn is None else vn
@@ -226,7 +227,7 @@ class StepBench:
             self.nact_log[i].copy_(s.n_active)
         for l in range(w.layers):
             s.kv_append(l, kn[l], vn[l])
-            s.decode_attn(l, q[l], self.out[l], w.softmax_scale)
+            s.decode_attn(l, q[l], out[l], w.softmax_scale)
 
     # ---- the method's own traffic (what one launch / one step must move) ----
     def algorithmic_bytes(self, steps):
@@ -352,14 +353,31 @@ def run_fdc(args, rank: int, world: int):
                     "frac_of_nominal_8TBs": round(achieved / NOMINAL_HBM_GBS, 4)}
 
         # pass 3: end to end through the C ABI with HOST buffers: every step copies its q / k_new /
-        # v_new from pinned host memory and reads the step's attention output back
+        # v_new from pinned host memory and reads the step's attention output back.  The copies run
+        # on a second stream with two sets of device buffers, so that the inputs of step i + 1 and the
+        # output of step i - 1 move while step i computes; all of them lie inside the timed region.
         e2e = None
         if with_e2e:
             hq_ = sb.q[W:].cpu().pin_memory()
             hk_ = sb.kn[W:].cpu().pin_memory()
             hv_ = sb.vn[W:].cpu().pin_memory()
             hout = torch.empty_like(sb.out, device="cpu").pin_memory()
-            dq, dk, dv = torch.empty_like(sb.q[0]), torch.empty_like(sb.kn[0]), torch.empty_like(sb.vn[0])
+            din = [(torch.empty_like(sb.q[0]), torch.empty_like(sb.kn[0]), torch.empty_like(sb.vn[0])) for _ in range(2)]
+            dout = [sb.out, torch.empty_like(sb.out)]
+            copies = torch.cuda.Stream(device)
+            in_ready = [ev() for _ in range(2)]      # inputs of a buffer set have arrived
+            computed = [ev() for _ in range(2)]      # the step that used a buffer set is done
+            out_read = [ev() for _ in range(2)]      # the output buffer has been copied to the host
+
+            def fetch(i):                            # on the copy stream: inputs of timed step i
+                b = i & 1
+                with torch.cuda.stream(copies):
+                    if i >= 2:
+                        copies.wait_event(computed[b])       # step i - 2 no longer reads this set
+                    for dst, src in zip(din[b], (hq_[i], hk_[i], hv_[i])):
+                        dst.copy_(src, non_blocking=True)
+                    in_ready[b].record(copies)
+
             sb.reset()
             for i in range(W):
                 sb.step(i)
@@ -368,16 +386,26 @@ def run_fdc(args, rank: int, world: int):
             torch.cuda.synchronize()
             e0, e1 = ev(), ev()
             e0.record(stream)
+            copies.wait_event(e0)
+            fetch(0)
             for i in range(K):
-                dq.copy_(hq_[i], non_blocking=True)
-                dk.copy_(hk_[i], non_blocking=True)
-                dv.copy_(hv_[i], non_blocking=True)
-                sb.step(W + i, dq, dk, dv)
-                hout.copy_(sb.out, non_blocking=True)
+                b = i & 1
+                if i + 1 < K:
+                    fetch(i + 1)
+                stream.wait_event(in_ready[b])
+                if i >= 2:
+                    stream.wait_event(out_read[b])           # the output of step i - 2 has left this buffer
+                sb.step(W + i, *din[b], out=dout[b])
+                computed[b].record(stream)
+                with torch.cuda.stream(copies):
+                    copies.wait_event(computed[b])
+                    hout.copy_(dout[b], non_blocking=True)
+                    out_read[b].record(copies)
+            stream.wait_stream(copies)                       # the last output is on the host
             e1.record(stream)
             torch.cuda.synchronize()
             ems = replicas.max_over_ranks(e0.elapsed_time(e1), device)
-            h2d = (dq.numel() + dk.numel() + dv.numel()) * w.esize
+            h2d = sum(t.numel() for t in din[0]) * w.esize
             d2h = sb.out.numel() * w.esize
             e2e = {"value": round(world * timed_bytes / (ems * 1e-3) / 1e9, 1), "unit": UNIT,
                    "ms_per_step": round(ems / K, 4), "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
