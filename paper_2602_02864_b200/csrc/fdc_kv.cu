@@ -23,8 +23,9 @@ __global__ void __launch_bounds__(128) kv_append_kernel(char* __restrict__ k, ch
     // Programmatic dependent launch.  The kernel after this one (the attention kernel) may be
     // scheduled as soon as every block of this grid is resident: its blocks then take the SMs as
     // they become free, set themselves up and wait for this grid to complete.  This grid waits for
-    // the kernel before it, so completion still follows the stream order.  The grid is small
-    // (at most n_slots blocks of 128 threads and few registers) so that all of it is resident early.
+    // the kernel before it, so completion still follows the stream order.  The grid is small (one
+    // block of 128 threads or two of 64 per SM at most, 32 registers a thread) so that all of it can
+    // be resident beside the attention blocks that are still running.
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     asm volatile("griddepcontrol.wait;" ::: "memory");
     // All loads of a slot are issued before anything depends on them (the rows of idle branch
