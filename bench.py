@@ -351,6 +351,11 @@ def run_fdc(args, rank: int, world: int):
                     # the tcgen05 kernel merges its partials itself: there is no combine launch to time
                     "combine_avg_launch_us": None if (w.dtype == "bf16" and w.head_dim == 128) else round(comb_ms / split_n * 1e3, 2),
                     "frac_of_nominal_8TBs": round(achieved / NOMINAL_HBM_GBS, 4)}
+            # the same launches inside the timed step loop (pass 1), where programmatic launches overlap
+            # the kernel before: region time / launches (frontier and build_masks included: < 1 %)
+            in_step_us = ms / split_n * 1e3
+            roof["avg_launch_us_in_step"] = round(in_step_us, 2)
+            roof["frac_in_step"] = round(avg_bytes / (in_step_us * 1e-6) / 1e9 / peak, 4)
 
         # pass 3: end to end through the C ABI with HOST buffers: every step copies its q / k_new /
         # v_new from pinned host memory and reads the step's attention output back.  The copies run
