@@ -346,3 +346,21 @@ def test_tile_list_that_breaks_the_prefix_rule_is_flagged():
     assert torch.equal(out[0], good[0])
     assert sess.status() == 0
     sess.close()
+
+
+@pytest.mark.parametrize("fused_append", [False, True], ids=["append_kernel", "append_inside_attention"])
+def test_more_pairs_than_thread_blocks(fused_append):
+    """40 scenes x 8 KV heads = 320 (scene, KV head) pairs for 148 thread blocks: every block then
+    works through several pairs (weighted split, a new set of queries per pair, whole pairs written
+    directly and cut ones merged), which the smaller cases never reach."""
+    w = wl.cfg4_sweep(512, 4, 40)
+    r = run_and_compare(w, check_steps={0, 1, 2, 31, 62, 63}, fused_append=fused_append)
+    assert r["steps"] == 64 and r["checked"] > 0
+
+
+@pytest.mark.parametrize("branches", [16, 32], ids=["64_query_rows", "128_query_rows"])
+def test_more_pairs_than_thread_blocks_wide(branches):
+    """The same regime with 64 and 128 query rows per pair (24 scenes x 8 KV heads = 192 pairs)."""
+    w = wl.cfg4_sweep(512, branches, 24)
+    r = run_and_compare(w, check_steps={0, 33, 63}, fused_append=True)
+    assert r["steps"] == 64 and r["checked"] > 0
