@@ -142,7 +142,7 @@ int fdc_plan_critical_path(const fdc_plan* plan, const int32_t* len, int32_t* st
  * rows after which field v of scene s is finished when no finish flag arrives earlier
  * (synthetic runs: the field's true length), or NULL to use the slot C[v] (truncation to the
  * fixed length, Sec. 3.3).  Values are clamped to [n_fixed+1, C]. */
-int fdc_state_init(const fdc_plan* plan, int32_t batch, const int32_t* d_len, void* d_state, void* stream);
+int fdc_state_init(fdc_plan* plan, int32_t batch, const int32_t* d_len, void* d_state, void* stream);
 
 /* Algorithm 1, one loop iteration (Sec. 3.2).  First retires the fields of the previous pass
  * that finished - branch slot b of scene s is finished if d_finish[s][b] != 0 (DEVICE uint8
@@ -157,7 +157,7 @@ int fdc_state_init(const fdc_plan* plan, int32_t batch, const int32_t* d_len, vo
  *   d_all_done int32 [1]                   1 iff no scene has a ready field left
  * A field admitted in this call decodes its first token in this pass; a field that finishes
  * in this pass is retired by the NEXT call.  All outputs are DEVICE memory. */
-int fdc_frontier(const fdc_plan* plan, int32_t batch, void* d_state, const uint8_t* d_finish,
+int fdc_frontier(fdc_plan* plan, int32_t batch, void* d_state, const uint8_t* d_finish,
                  int32_t* d_n_active, int32_t* d_node, int32_t* d_tok_idx, int32_t* d_kv_row,
                  int32_t* d_pos_id, int32_t* d_all_done, void* stream);
 
@@ -171,7 +171,7 @@ int fdc_frontier(const fdc_plan* plan, int32_t batch, void* d_state, const uint8
  *           ascending ids of the KV tiles (rows 64i..64i+63 of the scene's cache, prefix
  *           included) holding at least one row visible to some branch; 0 tiles for a scene
  *           with no active branch. */
-int fdc_build_masks(const fdc_plan* plan, int32_t batch, const void* d_state, uint64_t* d_mask,
+int fdc_build_masks(fdc_plan* plan, int32_t batch, const void* d_state, uint64_t* d_mask,
                     uint64_t* d_umask, int32_t* d_tiles, int32_t* d_ntiles, void* stream);
 
 /* Sec. 3.3 (shared KV cache, reused by all later passes): for every scene s and branch
@@ -180,7 +180,7 @@ int fdc_build_masks(const fdc_plan* plan, int32_t batch, const void* d_state, ui
  * skipped and flagged in the plan's status word.  d_k_new, d_v_new and d_kv_row are read for
  * every branch slot, idle ones included (the loads are issued before d_n_active is known), so
  * all of [batch][max_active] must be addressable; what idle slots hold does not matter. */
-int fdc_kv_append(const fdc_plan* plan, const fdc_kv_desc* kv, int32_t layer, const int32_t* d_n_active,
+int fdc_kv_append(fdc_plan* plan, const fdc_kv_desc* kv, int32_t layer, const int32_t* d_n_active,
                   const int32_t* d_kv_row, const void* d_k_new, const void* d_v_new, void* stream);
 
 /* Scratch for fdc_decode_attn (split partials); depends on the plan, the cache shape and the
@@ -203,7 +203,7 @@ int fdc_attn_workspace_bytes(const fdc_plan* plan, const fdc_kv_desc* kv, size_t
  * counters in the plan, and it leaves its work split there for the next call (checked against
  * d_n_active / d_ntiles before it is reused): calls that use the same plan must be ordered on
  * the GPU (one stream, or events); use one plan per concurrently decoding batch. */
-int fdc_decode_attn(const fdc_plan* plan, const fdc_kv_desc* kv, int32_t layer, const int32_t* d_n_active,
+int fdc_decode_attn(fdc_plan* plan, const fdc_kv_desc* kv, int32_t layer, const int32_t* d_n_active,
                     const uint64_t* d_mask, const int32_t* d_tiles, const int32_t* d_ntiles,
                     const void* d_q, void* d_out, float scale, void* d_workspace, size_t ws_bytes,
                     void* stream);
@@ -236,14 +236,14 @@ int fdc_decode_attn(const fdc_plan* plan, const fdc_kv_desc* kv, int32_t layer, 
  *     overlap on the GPU (different streams, or several host threads or plans on one device)
  *     race on it and corrupt each other's results: issue them on one stream or order them
  *     with events. */
-int fdc_decode_attn_static(const fdc_plan* plan, const fdc_kv_desc* kv, int32_t layer, const int32_t* d_n_active,
+int fdc_decode_attn_static(fdc_plan* plan, const fdc_kv_desc* kv, int32_t layer, const int32_t* d_n_active,
                            const uint64_t* d_mask, const int32_t* d_tiles, const int32_t* d_ntiles,
                            const void* d_q, void* d_out, float scale, void* stream);
 
 /* Reads (and with clear != 0 resets, together with the attention kernel's arrival counters,
  * which a launch that gave up may have left behind) the sticky device status word after
  * synchronising `stream`.  *host_bits receives the FDC_DEV_* bits; returns FDC_ERR_DEVICE if non-zero. */
-int fdc_status(const fdc_plan* plan, int32_t* host_bits, int32_t clear, void* stream);
+int fdc_status(fdc_plan* plan, int32_t* host_bits, int32_t clear, void* stream);
 
 /* Selects the split-pass kernel: 0 = automatic (3 for bf16, 1 for fp32), 1 = CUDA-core kernel
  * (any dtype), 2 = TMA + mma.sync kernel (bf16), 3 = TMA + tcgen05/TMEM kernel (bf16, head_dim

@@ -132,9 +132,9 @@ int fdc_plan_graph(const fdc_graph_desc* g, fdc_plan** out)
         p->sm_count = prop.multiProcessorCount;
         e = cudaMalloc((void**)&p->d, sizeof(PlanDev));
     }
-    if (e == cudaSuccess) e = cudaMalloc((void**)&p->d_status, (4 + FDC_PAIR_COUNTERS + 2 * FDC_MEMO_INTS) * sizeof(int32_t));
+    if (e == cudaSuccess) e = cudaMalloc((void**)&p->d_status, (4 + FDC_PAIR_COUNTERS + FDC_MEMO_INTS) * sizeof(int32_t));
     if (e == cudaSuccess) e = cudaMemcpy(p->d, &p->h, sizeof(PlanDev), cudaMemcpyHostToDevice);
-    if (e == cudaSuccess) e = cudaMemset(p->d_status, 0, (4 + FDC_PAIR_COUNTERS + 2 * FDC_MEMO_INTS) * sizeof(int32_t));
+    if (e == cudaSuccess) e = cudaMemset(p->d_status, 0, (4 + FDC_PAIR_COUNTERS + FDC_MEMO_INTS) * sizeof(int32_t));
     if (e != cudaSuccess) {
         int rc = set_cuda_error(e);
         fdc_plan_destroy(p);
@@ -143,7 +143,6 @@ int fdc_plan_graph(const fdc_graph_desc* g, fdc_plan** out)
     p->d_ticket = p->d_status + 2;
     p->d_pair_cnt = p->d_status + 4;
     p->d_split_memo = p->d_pair_cnt + FDC_PAIR_COUNTERS;
-    p->attn_seq = 0;
     p->fuse_append = 0;
     p->pend.valid = 0;
     *out = p;
@@ -221,7 +220,7 @@ int fdc_plan_critical_path(const fdc_plan* p, const int32_t* len, int32_t* steps
     return FDC_OK;
 }
 
-int fdc_status(const fdc_plan* p, int32_t* host_bits, int32_t clear, void* stream)
+int fdc_status(fdc_plan* p, int32_t* host_bits, int32_t clear, void* stream)
 {
     if (!p || !host_bits) return FDC_ERR_NULL;
     {

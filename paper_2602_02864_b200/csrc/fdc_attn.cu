@@ -128,7 +128,7 @@ const char* fdc_kernel_name(int32_t which)
     }
 }
 
-int fdc_decode_attn(const fdc_plan* p, const fdc_kv_desc* kv, int32_t layer, const int32_t* d_n_active,
+int fdc_decode_attn(fdc_plan* p, const fdc_kv_desc* kv, int32_t layer, const int32_t* d_n_active,
                     const uint64_t* d_mask, const int32_t* d_tiles, const int32_t* d_ntiles, const void* d_q,
                     void* d_out, float scale, void* d_workspace, size_t ws_bytes, void* stream)
 {
@@ -145,7 +145,7 @@ int fdc_decode_attn(const fdc_plan* p, const fdc_kv_desc* kv, int32_t layer, con
         const bool mine = takes_tc_kernel(p, kv) && app.kv.k == kv->k && app.kv.v == kv->v && app.layer == layer &&
                           app.stream == stream && app.d_n_active == d_n_active && app.kv.stride_layer == kv->stride_layer;
         if (mine) {
-            const_cast<fdc_plan*>(p)->pend.valid = 0;
+            p->pend.valid = 0;
         } else {
             rc = flush_pending_append(p);
             if (rc) return rc;
@@ -199,17 +199,50 @@ int fdc_decode_attn(const fdc_plan* p, const fdc_kv_desc* kv, int32_t layer, con
     a.pair_cnt = nullptr;
     a.split_memo = nullptr;
     a.seq = 0;
+    a.early = 0;
     bool fused = false;                 // the split kernel merged the partials itself
     if (kv->dtype == FDC_BF16 && (p->attn_kernel == 0 || p->attn_kernel == 3)) {
         if ((long long)kv->batch * kv->hkv <= FDC_PAIR_COUNTERS) a.pair_cnt = p->d_pair_cnt;
         a.split_memo = (a.pair_cnt && kv->batch <= FDC_MEMO_BATCH && a.n_cta <= FDC_MEMO_CTAS) ? p->d_split_memo : nullptr;
-        a.seq = ++const_cast<fdc_plan*>(p)->attn_seq;       // calls on one plan are ordered (see fdc.h)
+        // The work split depends only on the pass tables, so it is computed once per pass, by a launch
+        // of its own ahead of the pass's first attention launch (an ordinary launch: it begins after
+        // everything before it in the stream has completed).
+        bool split_now = false;
+        if (a.split_memo) {
+            const fdc_split_key& k = p->split_key;
+            split_now = !k.valid || k.tables_gen != p->tables_gen || k.d_n_active != d_n_active || k.d_ntiles != d_ntiles ||
+                        k.batch != kv->batch || k.hkv != kv->hkv || k.n_cta != a.n_cta || k.P != a.P || k.stream != stream;
+            if (split_now) {
+                a.seq = ++p->split_gen;
+                a.early = 0;
+                rc = launch_attn_tc_split(a, kv->head_dim, st);
+                if (rc == FDC_OK) {
+                    p->split_key = fdc_split_key{p->tables_gen, d_n_active, d_ntiles, kv->batch, kv->hkv, a.n_cta, a.P, stream, 1};
+                } else {
+                    p->split_key.valid = 0;
+                    a.split_memo = nullptr;
+                    split_now = false;
+                }
+                rc = FDC_ERR_SHAPE;
+            }
+            a.seq = p->split_gen;
+        }
+        // Reading ahead of the dependency wait: allowed from the second attention launch of a pass on
+        // the same stream.  The first one waits for everything before it (the pass tables, the split)
+        // before it lets the next kernel begin, and no kernel begins before the one ahead of it in the
+        // stream has let it, so whatever runs later finds those complete.
+        a.early = (!split_now && p->attn_gen == p->tables_gen && p->attn_stream == stream && p->attn_gen_valid) ? 1 : 0;
         if (app.valid) {
             a.app_row = app.d_kv_row;
             a.app_k = app.d_k_new;
             a.app_v = app.d_v_new;
         }
         rc = launch_attn_tc(a, kv->head_dim, st);
+        if (rc == FDC_OK) {
+            p->attn_gen = p->tables_gen;
+            p->attn_stream = stream;
+            p->attn_gen_valid = 1;
+        }
         a.app_row = nullptr;
         if (app.valid && rc != FDC_OK) {
             // the kernel that would have written the rows was not launched: append on its own after all

@@ -46,7 +46,7 @@ int static_ws_address(int device, void** out)
 
 }  // namespace
 
-extern "C" int fdc_decode_attn_static(const fdc_plan* p, const fdc_kv_desc* kv, int32_t layer,
+extern "C" int fdc_decode_attn_static(fdc_plan* p, const fdc_kv_desc* kv, int32_t layer,
                                       const int32_t* d_n_active, const uint64_t* d_mask, const int32_t* d_tiles,
                                       const int32_t* d_ntiles, const void* d_q, void* d_out, float scale,
                                       void* stream)

@@ -45,7 +45,7 @@ constexpr int TILE = FDC_TILE_ROWS;          // rows per entry of the visited-ti
 constexpr int RROWS = 2 * TILE;              // KV rows per round = M of S^T = K of O^T
 constexpr int NSOFT = 16;                    // softmax warps: 4 row quadrants x 4 column parts
 constexpr int NPART = NSOFT / 4;             // column parts
-constexpr int W_PROD = NSOFT, W_QK = NSOFT + 1, W_CLEAN = NSOFT + 2, W_PV = NSOFT + 3;
+constexpr int W_PROD = NSOFT, W_QK = NSOFT + 1, W_AUX = NSOFT + 2, W_PV = NSOFT + 3;
 constexpr int THREADS = (NSOFT + 4) * 32;
 constexpr uint32_t TMEM_COLS = 512;          // S^T buffers [0,256): 4 x 64 columns (2 x 128 for 128 query rows) | O^T [256,384) | sums [384,512)
 constexpr uint32_t TM_O = 256;
@@ -55,16 +55,21 @@ constexpr int STAGE = (D / 64) * PANEL;      // one K (or V) stage: 128 rows x h
 constexpr int MAXST = 4;                     // stages per ring at most
 constexpr float RAISE_LOG2 = 16.f;
 constexpr float UNSET = 1.0e30f;             // -reference of a column that has seen nothing yet
+#ifndef FDC_W_PREFIX
+#define FDC_W_PREFIX 4
+#endif
 #ifndef FDC_W_MASKED
-#define FDC_W_MASKED 3
+#define FDC_W_MASKED 6
 #endif
 #ifndef FDC_W_PAIR
-#define FDC_W_PAIR 8
+#define FDC_W_PAIR 32
 #endif
-constexpr int W_MASKED = FDC_W_MASKED;       // cost of a tile beyond the prefix (bitmap selects, V clean-up) in prefix tiles
+constexpr int W_PREFIX = FDC_W_PREFIX;       // cost of a tile inside the prefix (the unit of the weighted work split is a quarter of it)
+constexpr int W_MASKED = FDC_W_MASKED;       // cost of a tile beyond the prefix (bitmap selects, V clean-up): measured about 1.5 prefix tiles
 constexpr int W_PAIR = FDC_W_PAIR;           // cost of finishing a (scene, KV head) pair (drain, partial write, next queries)
 constexpr int UW = 64;                       // words of a scene's union bitmap kept in shared memory (when W <= UW)
-constexpr int MIN_UNITS = 8;                 // tiles per CTA below which fewer CTAs are used (small problems)
+constexpr int MIN_TILES = 8;                 // tiles per CTA below which fewer CTAs are used (small problems)
+constexpr int MIN_UNITS = MIN_TILES * W_PREFIX;   // the same as a weighted length
 static_assert(MIN_UNITS >= 2 * FDC_W_MASKED, "every part of a pair must contain the start of at least one tile");
 constexpr int MBUF = 512;                    // bitmap words of a scene kept in shared memory (max_active * W)
 
@@ -166,7 +171,7 @@ __device__ __forceinline__ float ord_to(int i) { return __int_as_float(i ^ ((i >
 
 // Everything a role needs to find its barriers and buffers.
 struct Ctx {
-    uint32_t k_full, k_empty, v_full, v_empty, v_clean, s_full, s_free, p_full, pv_done, q_ready, o_free, app_done;
+    uint32_t k_full, k_empty, v_full, v_empty, s_full, s_free, p_full, pv_done, q_ready, o_free, app_done;
     int ns, s_stride;                // S^T buffers in TMEM (4 of 64 columns up to 64 query rows, else 2 of 128) and their distance
     uint32_t tmem;
     unsigned char *kring, *vring, *qs, *ps;
@@ -183,7 +188,7 @@ struct Ctx {
     int npre;                        // tiles wholly inside the prefix
     long long vtot;                  // total weighted length
     volatile int* abortp;
-    volatile int* v_issued;          // V rounds the producer has requested so far (read by the cleaning warp)
+    volatile int* v_steps;           // [2][2] per P^T buffer and tile of the round: the 16-row steps to multiply (bit k: rows 16k..)
     int nk, nv, q_panel, p_buf, npb; // ring depths, bytes per 64-column panel of Q^T, bytes per P^T buffer, P^T buffers (1 or 2)
 };
 
@@ -210,19 +215,19 @@ __device__ __forceinline__ void cp_async_wait_all()
 
 // ---- weighted work split ---------------------------------------------------------------------
 // CTAs get equal shares of a WEIGHTED length, not of the tile count: a tile beyond the prefix
-// costs W_MASKED prefix tiles and the end of every pair costs W_PAIR.  Tile j of a pair starts at
+// costs W_MASKED / W_PREFIX prefix tiles and the end of every pair costs W_PAIR / W_PREFIX.  Tile j of a pair starts at
 // weighted offset vt(j); a pair of nt tiles is vt(nt) + W_PAIR long.  A CTA owns the tiles whose
 // start falls into its share, so shares always cut the unit sequence into consecutive runs.
 __device__ __forceinline__ int vt_of(const Ctx& cx, int nt, int j)
 {
     const int np = cx.npre < nt ? cx.npre : nt;
-    return j <= np ? j : np + (j - np) * W_MASKED;
+    return j <= np ? j * W_PREFIX : np * W_PREFIX + (j - np) * W_MASKED;
 }
 // First tile of a pair of nt tiles whose weighted start is >= r (nt if there is none).
 __device__ __forceinline__ int tile_of_vt(const Ctx& cx, int nt, int r)
 {
     const int np = cx.npre < nt ? cx.npre : nt;
-    const int j = r <= np ? r : np + (r - np + W_MASKED - 1) / W_MASKED;
+    const int j = r <= np * W_PREFIX ? (r + W_PREFIX - 1) / W_PREFIX : np + (r - np * W_PREFIX + W_MASKED - 1) / W_MASKED;
     return j > nt ? nt : j;
 }
 // First unit whose weighted start is >= x.
@@ -274,7 +279,9 @@ struct Cursor {
 __device__ __forceinline__ void cursor_batch(Cursor& c, const AttnParams& p, int lane)
 {
     c.jn = c.sg.j1 - c.jb < 32 ? c.sg.j1 - c.jb : 32;
-    c.my_tile = lane < c.jn ? p.tiles[(size_t)c.sg.s * p.ntile_max + c.jb + lane] : 0;
+    // entry j of a tile list is tile j for every whole tile of the prefix: no need to read those
+    const int j = c.jb + lane;
+    c.my_tile = lane < c.jn ? (j < p.P / TILE ? j : p.tiles[(size_t)c.sg.s * p.ntile_max + j]) : 0;
     c.k = 0;
 }
 __device__ __forceinline__ void cursor_open(Cursor& c, const AttnParams& p, const Ctx& cx, long long hi, int lane)
@@ -342,13 +349,24 @@ __device__ __forceinline__ void producer_loop(const AttnParams& p, const Ctx& cx
     int ok = 1;
     uint32_t idle = 0;
     int app_ok = p.app_row == nullptr;               // rows appended by this kernel are in place (tiles beyond the prefix may be loaded)
+    int waited = !p.early;                           // the kernel ahead in the stream has completed (griddepcontrol.wait was taken)
+    int q_hold = p.early;                            // after the wait, the first pair's queries go ahead of further K/V requests
     while ((ck.live || cv.live) && ok) {
-        if (!app_ok) {
+        if (!app_ok && waited) {
             const int done = lane == 0 ? (int)mbar_try(cx.app_done, 0) : 0;
             app_ok = __shfl_sync(0xffffffffu, done, 0);
         }
-        const bool hold_k = !app_ok && ck.live && cursor_beyond_prefix(ck, p.P);
-        const bool hold_v = !app_ok && cv.live && cursor_beyond_prefix(cv, p.P);
+        // Rows beyond the prefix may have been written by the kernel ahead (fdc_kv_append) or are written
+        // by this one (fused append): their tiles wait for both.  Prefix rows never change during decode.
+        if (q_hold && waited) {
+            // The queries are requested right after the wait; whatever this SM requests before them
+            // arrives before them.  The stages requested ahead of the wait keep the first rounds fed.
+            const int done = lane == 0 ? (int)mbar_try(cx.q_ready, 0) : 0;
+            q_hold = !__shfl_sync(0xffffffffu, done, 0);
+        }
+        const bool hold_all = q_hold && waited;
+        const bool hold_k = hold_all || (!(app_ok && waited) && ck.live && cursor_beyond_prefix(ck, p.P));
+        const bool hold_v = hold_all || (!(app_ok && waited) && cv.live && cursor_beyond_prefix(cv, p.P));
         int rk = 0, rv = 0;
         if (lane == 0) {
             rk = ck.live && !hold_k && mbar_try(cx.k_empty + 8 * ck.st, ck.ph ^ 1);
@@ -362,11 +380,14 @@ __device__ __forceinline__ void producer_loop(const AttnParams& p, const Ctx& cx
         }
         if (rv) {
             cursor_issue(cv, tm_v, cx.vring, cx.v_full, pol, lane);
-            if (lane == 0) *cx.v_issued = (int)cv.g + 1;
             cursor_next(cv, p, cx, hi, cx.nv, lane);
         }
         if (rk | rv) {
             idle = 0;
+        } else if (!waited) {
+            // nothing more can be requested ahead of the kernel before this one: wait for it to complete
+            asm volatile("griddepcontrol.wait;" ::: "memory");
+            waited = 1;
         } else if (((++idle) & 63u) == 0u) {
             // bounded: no stage became free for a long time, or another role gave up
             if (idle >= SPIN_LIMIT) {
@@ -382,6 +403,7 @@ __device__ __forceinline__ void producer_loop(const AttnParams& p, const Ctx& cx
             }
         }
     }
+    if (!waited) asm volatile("griddepcontrol.wait;" ::: "memory");     // (a run wholly inside the prefix that fitted the rings)
     if (!ok && lane == 0) {
         // give the copies already in flight a bounded chance to land before the CTA ends
         for (int r = 0; r < 2; ++r) {
@@ -448,51 +470,6 @@ __device__ __forceinline__ void qk_loop(const AttnParams& p, const Ctx& cx, long
     }
 }
 
-// V rows of a stage that are invisible to every branch of the scene are cleared (whole warp; kept
-// out of line: only rounds beyond the prefix come here).  tile0 / tile1 are the round's tiles, vs
-// the stage's shared-memory address.  `un` is the OR of the scene's bitmaps when the softmax warps
-// have prepared it (the usual case), else nullptr and the bitmaps themselves are combined here.
-__device__ __noinline__ void clear_unseen_rows(uint32_t vs, const uint64_t* un, const uint64_t* mask0, int W, int P, int A, int tile0, int tile1, int nt)
-{
-    const int lane = threadIdx.x & 31;
-    bool touched = false;
-    for (int i = 0; i < nt; ++i) {
-        const int tile = i ? tile1 : tile0;
-        if (tile * TILE + TILE <= P) continue;                 // all rows visible to everybody
-        uint64_t seen;
-        if (un) {
-            seen = tile_rowmask(un, W, P, tile);
-        } else {
-            uint64_t um = 0ull;
-            for (int b = lane; b < A; b += 32) um |= tile_rowmask(mask0 + (size_t)b * W, W, P, tile);
-            const uint32_t ul = __reduce_or_sync(0xffffffffu, (uint32_t)um);
-            const uint32_t uh = __reduce_or_sync(0xffffffffu, (uint32_t)(um >> 32));
-            seen = ((uint64_t)uh << 32) | ul;
-        }
-        const uint64_t z = ~seen;
-        if (z) {
-            // lane l clears rows l and l + 32 of the tile if nobody sees them (2 panels x 8 chunks of 16 bytes)
-#pragma unroll
-            for (int hr = 0; hr < 2; ++hr) {
-                const int r = lane + 32 * hr;
-                if ((z >> r) & 1) {
-                    const uint32_t row = vs + (i * TILE + r) * 128;
-#pragma unroll
-                    for (int ch = 0; ch < 8; ++ch) {
-                        // rotate the chunk order by the row so that the lanes of a warp hit different banks
-                        const uint32_t cc = ((ch + r) & 7) << 4;
-                        asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(row + cc), "r"(0u) : "memory");
-                        asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(row + PANEL + cc), "r"(0u) : "memory");
-                    }
-                }
-            }
-            touched = true;
-        }
-    }
-    if (touched) fence_async_smem();
-    __syncwarp();
-}
-
 // Fused append (one warp; out of line, all arguments by value).  The new K/V vectors of this pass
 // (Sec. 3.3: every emitted token's K/V is written once, at the row its slot reserves) whose rows
 // lie in KV tiles that this CTA owns are written here, before the CTA loads those tiles: every
@@ -550,100 +527,45 @@ __device__ __noinline__ void append_rows(char* kc, char* vc, long long stride_sc
     __syncwarp();
 }
 
-// Bounded wait until the producer has requested V round g (*issued > g).
-__device__ __noinline__ int wait_issued(volatile int* issued, int g, volatile int* abort_flag, int32_t* status)
+// Rows of a KV tile beyond the prefix that some branch of the scene may see (the OR of the
+// branches' bitmaps; prefix rows of a tile that straddles the end of the prefix included).  `un` is
+// that OR as the softmax warps prepared it per pair (the usual case), else nullptr and the bitmaps
+// themselves are combined here (templates too long for the shared-memory copy).
+__device__ __noinline__ uint64_t tile_seen_rows(const uint64_t* un, const uint64_t* mask0, int W, int P, int A, int tile)
 {
-    for (uint32_t i = 0; i < SPIN_LIMIT; ++i) {
-        if (*issued > g) return 1;
-        if (*abort_flag) return 0;
-        __nanosleep(64);
-    }
-    *abort_flag = 1;
-    atomicOr(status, FDC_DEV_TIMEOUT);
-    return 0;
+    if (un) return tile_rowmask(un, W, P, tile);
+    uint64_t um = 0ull;
+    for (int b = 0; b < A; ++b) um |= tile_rowmask(mask0 + (size_t)b * W, W, P, tile);
+    return um;
 }
 
-// One warp: the V rows of a stage that are invisible to every branch of the scene are cleared
-// before the stage is multiplied.  Their P^T row is exactly 0, but the rows can hold anything
-// (NaN, Inf: slots that were never written) and 0 * NaN must not reach the accumulator.  Stages
-// wholly inside the prefix are passed on as they are.  A warp of its own, so that the clean-up
-// runs ahead (as far as the V ring is deep) instead of delaying the multiplications.
-__device__ __forceinline__ void clean_loop(const AttnParams& p, const Ctx& cx, long long lo, long long hi, int lane)
+// The auxiliary warp: with fdc_set_fused_append it writes the pass's new K/V rows that fall into
+// this CTA's tiles, then lets the producer go on to the tiles beyond the prefix.
+__device__ __forceinline__ void aux_loop(const AttnParams& p, const Ctx& cx, long long lo, long long hi, int lane)
 {
     if (p.app_row) {
-        // a recorded fdc_kv_append: this warp writes the rows that fall into the CTA's tiles, then lets
-        // the producer go on to the tiles beyond the prefix
         append_rows(const_cast<char*>(reinterpret_cast<const char*>(p.k)), const_cast<char*>(reinterpret_cast<const char*>(p.v)),
                     p.stride_scene * 2, p.stride_head * 2, p.stride_row * 2, p.app_row, reinterpret_cast<const char*>(p.app_k),
                     reinterpret_cast<const char*>(p.app_v), p.tiles, p.ntile_max, p.max_active, p.hkv, p.rows, p.P, cx.pre, cx.nact, lo, hi,
                     p.status);
         if (lane == 0) mbar_arrive(cx.app_done);
     }
-    int s = 0;
-    uint32_t seg = 0, g = 0;
-    int st = 0;
-    uint32_t vph = 0;
-    long long u = lo;
-    int ok = 1;
-    while (u < hi && ok) {
-        const Segment sg = decode_segment(u, hi, cx.pre, p.hkv, s);
-        const int A = cx.nact[sg.s];
-        bool have_masks = !cx.mstaged;                 // staged bitmaps are published with the queries (q_ready)
-        for (int jb = sg.j0; jb < sg.j1 && ok; jb += 32) {
-            const int jn = sg.j1 - jb < 32 ? sg.j1 - jb : 32;
-            const int my_tile = lane < jn ? p.tiles[(size_t)sg.s * p.ntile_max + jb + lane] : 0;
-            for (int k = 0; k < jn && ok; k += 2, ++g) {
-                const int nt = jn - k < 2 ? 1 : 2;
-                // tile ids ascend: the round reaches beyond the prefix iff its last tile does
-                const int t_last = __shfl_sync(0xffffffffu, my_tile, (k + nt - 1) & 31);
-                const bool masked = t_last * TILE + TILE > p.P;
-                // Which rounds pass through this warp is decided by POSITION on both sides (entry j of a list
-                // is tile j inside the prefix), so the two can never disagree about the barrier; a list that
-                // breaks the rule is flagged (an uncleaned stage could have been multiplied).
-                const bool beyond = jb + k + nt - 1 >= p.P / TILE;
-                if (lane == 0 && masked != beyond) atomicOr(p.status, FDC_DEV_TILE_LIST);
-                if (beyond) {
-                    int okw = 1;
-                    if (lane == 0) {
-                        // Rounds inside the prefix are skipped without a wait, so this warp can be far ahead of
-                        // the ring: it first waits until the producer has requested round g (then the stage's
-                        // barrier cannot be in an earlier phase with the same parity), then for the data.
-                        okw = wait_issued(cx.v_issued, (int)g, cx.abortp, p.status);
-                        if (okw) okw = mbar_wait(cx.v_full + 8 * st, vph, cx.abortp, p.status);
-                        if (okw && masked && !have_masks) okw = mbar_wait(cx.q_ready, seg & 1, cx.abortp, p.status);
-                    }
-                    ok = __shfl_sync(0xffffffffu, okw, 0);
-                    if (ok && masked) {
-                        have_masks = true;
-                        clear_unseen_rows(smem_u32(cx.vring) + st * STAGE, (cx.mstaged && p.W <= UW) ? cx.sunion + (seg & 1) * UW : nullptr,
-                                          mask_row(p, cx, seg, sg.s, 0), p.W, p.P, A, __shfl_sync(0xffffffffu, my_tile, k & 31), t_last, nt);
-                    }
-                    if (ok && lane == 0) mbar_arrive(cx.v_clean + 8 * st);
-                }
-                if (++st == cx.nv) {
-                    st = 0;
-                    vph ^= 1;
-                }
-            }
-        }
-        ++seg;
-        u = sg.next_u;
-    }
 }
 
-// One elected thread: O^T += V^T(stage) P^T[g & 1] for every round g, once the stage has been
-// passed on by the cleaning warp and the softmax warps have delivered P^T.
+// One elected thread: O^T += V^T(stage) P^T[g & 1] for every round g, once the stage has landed and
+// the softmax warps have delivered P^T (and, beyond the prefix, cleared the stage's unseen rows).
+// The multiplication runs in steps of 16 KV rows; the softmax warps say which steps hold a visible
+// row (all of them inside the prefix), the others are left out.
 __device__ __forceinline__ void pv_loop(const AttnParams& p, const Ctx& cx, long long lo, long long hi, int lane)
 {
     const uint64_t v_desc0 = smem_desc(smem_u32(cx.vring), PANEL, 1024);
     const uint64_t p_desc0 = smem_desc(smem_u32(cx.ps), PANEL, 1024);
     const uint32_t v_lo0 = (uint32_t)v_desc0, v_hi = (uint32_t)(v_desc0 >> 32), p_lo0 = (uint32_t)p_desc0, p_hi = (uint32_t)(p_desc0 >> 32);
     const uint32_t tm_o = cx.tmem + TM_O;
-    const int npre_tiles = p.P / TILE;
     int s = 0;
     uint32_t g = 0, seg = 0;
     int st = 0;
-    uint32_t vph = 0, cpar = 0;
+    uint32_t vph = 0;
     long long u = lo;
     int ok = 1;
     while (u < hi && ok) {
@@ -655,29 +577,27 @@ __device__ __forceinline__ void pv_loop(const AttnParams& p, const Ctx& cx, long
             const int ntile = sg.j1 - sg.j0;
             bool good = true;
             for (int t = 0; 2 * t < ntile && good; ++t, ++g) {
-                const int nt = ntile - 2 * t < 2 ? 1 : 2;
-                // Entry j of a tile list is tile j for every whole prefix tile, so the position tells whether
-                // the round reaches beyond the prefix.  Only then does the stage come through the cleaning
-                // warp (which may still be busy with the append at the start of the CTA); v_clean[st]
-                // completes one phase per such round, counted in cpar on both sides.
-                const bool beyond = sg.j0 + 2 * t + nt - 1 >= npre_tiles;
-                if (beyond) {
-                    good = mbar_wait(cx.v_clean + 8 * st, (cpar >> st) & 1u, cx.abortp, p.status);
-                    cpar ^= 1u << st;
-                } else {
-                    good = mbar_wait(cx.v_full + 8 * st, vph, cx.abortp, p.status);
-                }
+                good = mbar_wait(cx.v_full + 8 * st, vph, cx.abortp, p.status);
                 if (good) good = mbar_wait(cx.p_full + 8 * (g & 1), (g >> 1) & 1, cx.abortp, p.status);
                 if (good && t == 0 && seg > 0) good = mbar_wait(cx.o_free, (seg - 1) & 1, cx.abortp, p.status);
                 if (!good) break;
+                const uint32_t steps = (uint32_t)cx.v_steps[(g & 1) * 2] | ((uint32_t)cx.v_steps[(g & 1) * 2 + 1] << 4);
                 tc_fence_after();
                 const uint32_t vd = v_lo0 + (uint32_t)((st * STAGE) >> 4);
                 const uint32_t pd = p_lo0 + (uint32_t)((((g & 1) & (cx.npb - 1)) * cx.p_buf) >> 4);
+                if (steps == 0xffu) {
 #pragma unroll
-                for (int kk = 0; kk < 4; ++kk) umma2(tm_o, vd + kk * 128, v_hi, pd + kk * 128, p_hi, idesc_pv, (t > 0 || kk > 0) ? 1u : 0u);
-                if (nt == 2) {                                       // a one-tile round has 64 KV rows
-#pragma unroll
-                    for (int kk = 4; kk < 8; ++kk) umma2(tm_o, vd + kk * 128, v_hi, pd + kk * 128, p_hi, idesc_pv, 1u);
+                    for (int kk = 0; kk < 8; ++kk) umma2(tm_o, vd + kk * 128, v_hi, pd + kk * 128, p_hi, idesc_pv, (t > 0 || kk > 0) ? 1u : 0u);
+                } else {
+                    // a one-tile round has 64 KV rows; beyond the prefix, steps without a visible row are left out
+                    // (rows that nobody may see can hold NaN, and 0 * NaN must not reach the accumulator)
+                    uint32_t acc = t > 0 ? 1u : 0u;
+#pragma unroll 1
+                    for (int kk = 0; kk < 8; ++kk)
+                        if ((steps >> kk) & 1u) {
+                            umma2(tm_o, vd + kk * 128, v_hi, pd + kk * 128, p_hi, idesc_pv, acc);
+                            acc = 1u;
+                        }
                 }
                 umma_commit(cx.v_empty + 8 * st);
                 umma_commit(cx.pv_done + 8 * (g & 1));
@@ -692,34 +612,29 @@ __device__ __forceinline__ void pv_loop(const AttnParams& p, const Ctx& cx, long
         g = __shfl_sync(0xffffffffu, g, 0);
         st = __shfl_sync(0xffffffffu, st, 0);
         vph = __shfl_sync(0xffffffffu, vph, 0);
-        cpar = __shfl_sync(0xffffffffu, cpar, 0);
         ++seg;
         u = sg.next_u;
     }
 }
 
-// Visibility (Eq. 1) of one KV row for the nph query columns starting at col0: bit i <=> column
-// col0 + i may see the row.  The warp's 32 rows are rows 32 * upper .. of tile `tile`; lane b first
-// extracts the rows' bits of branch b (and b + 32), then every lane collects its own row's bit of
-// the branches its columns belong to.  Kept out of line: only tiles beyond the prefix need it.
-__device__ __noinline__ uint64_t row_visibility(const uint64_t* mask0, int W, int P, int tile, int A, int G, int col0, int nph, int upper)
+// Visibility (Eq. 1) of one KV row for the nph (<= 32) query columns starting at col0: bit i <=>
+// column col0 + i may see the row.  `row` (0..63) is the thread's row inside tile `tile`.  Columns
+// b * G .. b * G + G - 1 belong to branch b; every thread reads the bitmap words of the two or three
+// branches its columns belong to (the same words for the whole warp: one broadcast read each).
+// When the prefix is a whole number of tiles a tile's 64 rows are one word of the bitmap; otherwise
+// they straddle two (tile_rowmask).  Only tiles beyond the prefix come here.
+__device__ __forceinline__ uint32_t row_visibility(const uint64_t* mask0, int W, int P, int tile, int row, int A, int G, int b_lo, int col0, int nph)
 {
-    const int lane = threadIdx.x & 31;
-    uint64_t m0 = 0ull, m1 = 0ull;
-    if (lane < A) m0 = tile_rowmask(mask0 + (size_t)lane * W, W, P, tile);
-    if (lane + 32 < A) m1 = tile_rowmask(mask0 + (size_t)(lane + 32) * W, W, P, tile);
-    const uint32_t wlo = upper ? (uint32_t)(m0 >> 32) : (uint32_t)m0;
-    const uint32_t whi = upper ? (uint32_t)(m1 >> 32) : (uint32_t)m1;
-    uint64_t vis = 0ull;
-    const int b_lo = col0 / G, b_hi = (col0 + nph - 1) / G;
-    for (int bq = b_lo; bq <= b_hi; ++bq) {
-        const uint32_t bits = __shfl_sync(0xffffffffu, bq < 32 ? wlo : whi, bq & 31);
-        if ((bits >> lane) & 1) {
-            const int c_lo = bq * G - col0 < 0 ? 0 : bq * G - col0;
-            const int c_hi = (bq + 1) * G - col0 > nph ? nph : (bq + 1) * G - col0;     // exclusive
-            const uint64_t span = c_hi - c_lo == 64 ? ~0ull : ((1ull << (c_hi - c_lo)) - 1ull);
-            vis |= span << c_lo;
-        }
+    uint32_t vis = 0u;
+    const bool aligned = (P & (TILE - 1)) == 0;
+    const int w = tile - P / TILE;
+    int c = b_lo * G - col0;                       // first column of branch b relative to col0 (<= 0 for the first one)
+#pragma unroll 1
+    for (int b = b_lo; b < A && c < nph; ++b, c += G) {
+        const uint64_t word = aligned ? (w < W ? mask0[(size_t)b * W + w] : 0ull) : tile_rowmask(mask0 + (size_t)b * W, W, P, tile);
+        const int lo = c < 0 ? 0 : c, hi = c + G > nph ? nph : c + G;
+        const uint32_t span = (hi - lo >= 32 ? 0xffffffffu : ((1u << (hi - lo)) - 1u)) << lo;
+        if ((word >> row) & 1ull) vis |= span;
     }
     return vis;
 }
@@ -746,6 +661,34 @@ __device__ __noinline__ void prefetch_next_segment(const uint4* qg, const uint64
     if (smask_dst) {
         const uint64_t* src = mask + (size_t)nx.s * max_active * W;
         for (int idx = tid; idx < max_active * W; idx += NSOFT * 32) cp_async8(smask_dst + idx, src + idx);
+    }
+}
+
+// The first pair's bitmaps and queries when the kernel runs ahead of the dependency wait (softmax
+// threads; out of line, arguments by value).  The bitmaps are complete and are copied right away.
+// The queries may still be written by the kernel ahead: their lines are only requested into L2
+// (which stays coherent), the wait is taken, and then they are read and laid out as Q^T.
+__device__ __noinline__ void stage_first_pair_early(const uint4* qg, const uint64_t* mask, int max_active, int W, int hq, int G, int s, int g, int M,
+                                                    unsigned char* qs, int q_panel, uint64_t* smask_dst)
+{
+    const int tid = threadIdx.x;
+    const int NP = M <= 32 ? 32 : (M <= 64 ? 64 : 128);
+    if (smask_dst) {
+        const uint64_t* src = mask + (size_t)s * max_active * W;
+        for (int idx = tid; idx < max_active * W; idx += NSOFT * 32) smask_dst[idx] = src[idx];
+    }
+    for (int idx = tid * 8; idx < M * (D / 8); idx += NSOFT * 32 * 8) {      // one request per 128-byte line
+        const int n = idx / (D / 8), ch = idx - n * (D / 8);
+        const int bb = n / G, hg = n - bb * G;
+        asm volatile("prefetch.global.L2 [%0];" ::"l"(qg + ((((size_t)s * max_active + bb) * hq + (size_t)g * G + hg) * D) / 8 + ch));
+    }
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    for (int idx = tid; idx < NP * (D / 8); idx += NSOFT * 32) {
+        const int n = idx / (D / 8), ch = idx - n * (D / 8);
+        const bool valid = n < M;
+        const int bb = valid ? n / G : 0, hg = valid ? n - bb * G : 0;
+        cp_async16(qs + (ch >> 3) * q_panel + n * 128 + (((ch & 7) ^ (n & 7)) << 4),
+                   qg + ((((size_t)s * max_active + bb) * hq + (size_t)g * G + hg) * D) / 8 + ch, valid);
     }
 }
 
@@ -820,7 +763,7 @@ struct RaiseArgs {
     int32_t* status;
     uint32_t s_addr, o_addr, l_addr;   // TMEM addresses of this thread's first score / accumulator / sum column
     uint32_t pv_bar, pv_parity;  // completion of the previous round's O^T += V^T P^T
-    uint64_t vis;                // Eq. 1 bits of this thread's columns
+    uint32_t vis;                // Eq. 1 bits of this thread's columns
     float c;
     int col0, nph, live, rescale_o, dead;
 };
@@ -839,7 +782,7 @@ __device__ __noinline__ int raise_references(const RaiseArgs a)
             tmem_ld<8>(a.s_addr + ch * 8, sv);
             tmem_wait_ld();
             float v[8];
-            const uint32_t vb = (uint32_t)(a.vis >> (ch * 8));
+            const uint32_t vb = a.vis >> (ch * 8);
 #pragma unroll
             for (int i = 0; i < 8; ++i) v[i] = ((vb >> i) & 1) ? __uint_as_float(sv[i]) * a.c : -INFINITY;
             // lanes whose index differs in bits >= 8 hold rows of the same columns: plain max
@@ -923,7 +866,7 @@ __device__ __noinline__ int raise_references(const RaiseArgs a)
 // TMEM (the free columns [384, 512)) and the references read from shared memory, so that the
 // same small loop serves every width.
 __device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& cx, const Segment& sg, const int nph, const uint32_t seg,
-                                                const long long hi, int& prefetched, uint32_t& g, bool& dead, const int warp, const int lane)
+                                                const long long hi, int& prefetched, uint32_t& g, int& vst, uint32_t& vph, bool& dead, const int warp, const int lane)
 {
     const int np = NPART * nph, nch = nph >> 3;
     const int tid = threadIdx.x;                  // 0..NSOFT * 32 - 1
@@ -935,6 +878,7 @@ __device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& 
     const int A = cx.nact[sg.s];
     const int M = A * p.group;
     const int G = p.group;
+    const int b_lo = col0 / G;                    // branch of this thread's first query column
     const uint32_t o_addr = cx.tmem + lane_base + TM_O + col0;
     const uint32_t l_addr = cx.tmem + lane_base + TM_L + col0;
     auto wait_u = [&](uint32_t bar, uint32_t parity) {    // warp-uniform outcome
@@ -983,7 +927,7 @@ __device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& 
             }
         }
         if (cx.mstaged && p.W <= UW) {
-            // OR of the scene's bitmaps: the rows no branch may see, for the warp that cleans V
+            // OR of the scene's bitmaps: the rows that some branch may see (the others are cleared in V)
             soft_sync();                              // everybody's share of the bitmaps is in place
             if (tid < p.W) {
                 const uint64_t* mb = cx.smask + (seg & 1) * MBUF + tid;
@@ -1019,7 +963,7 @@ __device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& 
             const bool live = ti < nt && !dead;                       // rows 64..127 of a one-tile round hold nothing
             const bool masked = live && tile * TILE + TILE > p.P;
             // Eq. 1 for this thread's KV row: bit i of vis <=> column col0 + i may see the row
-            const uint64_t vis = masked ? row_visibility(mask_row(p, cx, seg, sg.s, 0), p.W, p.P, tile, A, G, col0, nph, q4 & 1) : ~0ull;
+            const uint32_t vis = masked ? row_visibility(mask_row(p, cx, seg, sg.s, 0), p.W, p.P, tile, (q4 & 1) * 32 + lane, A, G, b_lo, col0, nph) : ~0u;
             const uint32_t sb = g & (cx.ns - 1);                      // score buffer of the round
             wait_u(cx.s_full + 8 * sb, (g / cx.ns) & 1);
             tc_fence_after();
@@ -1089,7 +1033,7 @@ __device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& 
                     const float mn[8] = {m0.x, m0.y, m0.z, m0.w, m1.x, m1.y, m1.z, m1.w};
                     tmem_wait_ld();
                     if (masked) {                                      // uniform branch: prefix rounds skip the selects
-                        const uint32_t vb = (uint32_t)(vis >> (ch * 8));
+                        const uint32_t vb = vis >> (ch * 8);
 #pragma unroll
                         for (int i = 0; i < 8; ++i)
                             if (!((vb >> i) & 1)) sv[i] = 0xff800000u;
@@ -1120,6 +1064,39 @@ __device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& 
                     cx.rflag[g & 3] = (int)g;
                     if (!(emax < 1.0e30f)) atomicOr(p.status, FDC_DEV_SCORE_RANGE);     // beyond 2^100 (or inf / nan)
                 }
+            }
+            // ---- this round's V stage.  Beyond the prefix, rows that no branch of the scene may see can hold
+            // anything (NaN, Inf: slots that were never written), and although their P^T entries are
+            // exactly 0, 0 * NaN must not reach the accumulator.  The multiplication runs in steps of 16
+            // KV rows: a step without any visible row is left out, and in the other steps the unseen
+            // rows are cleared here, every thread a quarter of its own row, once the stage has landed.
+            uint32_t st4 = live ? 0xfu : 0u;                           // steps of this warp's tile to multiply
+            if (masked) {                                              // (uniform over the warp)
+                const uint64_t* un = (cx.mstaged && p.W <= UW) ? cx.sunion + (seg & 1) * UW : nullptr;
+                const int w = tile - p.P / TILE;
+                const uint64_t seen = (un && (p.P & (TILE - 1)) == 0) ? (w < p.W ? un[w] : 0ull)
+                                                                       : tile_seen_rows(un, mask_row(p, cx, seg, sg.s, 0), p.W, p.P, A, tile);
+                wait_u(cx.v_full + 8 * vst, vph);
+                const int row = (q4 & 1) * 32 + lane;
+                const bool none = seen == 0ull;                        // (such a tile should not be listed: clear and multiply all of it)
+                const uint32_t step_seen = (uint32_t)(seen >> (row & 48)) & 0xffffu;
+                if (!dead && (none || (step_seen != 0u && !((seen >> row) & 1ull)))) {
+                    const uint32_t va = smem_u32(cx.vring) + (uint32_t)vst * STAGE + (uint32_t)(part >> 1) * PANEL +
+                                        (uint32_t)(ti * TILE + row) * 128 + (uint32_t)(part & 1) * 64;
+#pragma unroll
+                    for (int i = 0; i < 4; ++i)
+                        asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(va + (uint32_t)((i + lane) & 3) * 16), "r"(0u) : "memory");
+                }
+                st4 = 0u;
+#pragma unroll
+                for (int i = 0; i < 4; ++i) st4 |= (none || ((seen >> (16 * i)) & 0xffffull)) ? (1u << i) : 0u;
+                // the whole tiles of the prefix come first in a tile list (entry j = tile j): the producer relies on it
+                if (part == 0 && (q4 & 1) == 0 && lane == 0 && sg.j0 + jb + k + ti < p.P / TILE) atomicOr(p.status, FDC_DEV_TILE_LIST);
+            }
+            if (part == 0 && (q4 & 1) == 0 && lane == 0) cx.v_steps[b * 2 + ti] = (int)st4;
+            if (++vst == cx.nv) {
+                vst = 0;
+                vph ^= 1;
             }
             // every thread orders its own TMEM reads and shared-memory writes, then one lane per warp signals
             tc_fence_before();
@@ -1235,7 +1212,7 @@ __device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& 
 
 __global__ void __launch_bounds__(THREADS, 1)
 attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
-               const int nk, const int nv, const int np_max, const int npb)
+               const int nk, const int nv, const int np_max, const int npb, const int split_only)
 {
     extern __shared__ unsigned char smem_dyn[];
     unsigned char* smem = reinterpret_cast<unsigned char*>(((uintptr_t)smem_dyn + 1023) & ~(uintptr_t)1023);
@@ -1254,8 +1231,7 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, con
     cx.k_empty = cx.k_full + 8 * MAXST;
     cx.v_full = cx.k_empty + 8 * MAXST;
     cx.v_empty = cx.v_full + 8 * MAXST;
-    cx.v_clean = cx.v_empty + 8 * MAXST;
-    cx.s_full = cx.v_clean + 8 * MAXST;
+    cx.s_full = cx.v_empty + 8 * MAXST;
     cx.s_free = cx.s_full + 8 * 4;
     cx.p_full = cx.s_free + 8 * 4;
     cx.ns = np_max <= 64 ? 4 : 2;
@@ -1277,16 +1253,45 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, con
     cx.smask = reinterpret_cast<uint64_t*>(((uintptr_t)(cx.prev + p.batch + 1) + 7) & ~(uintptr_t)7);
     cx.sunion = cx.smask + 2 * MBUF;
     cx.mstaged = p.max_active * p.W <= MBUF;
-    __shared__ int abort_flag, v_issued_count;
+    __shared__ int abort_flag, v_step_bits[4];
     cx.abortp = &abort_flag;
-    cx.v_issued = &v_issued_count;
+    cx.v_steps = v_step_bits;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 0) {
         abort_flag = 0;
-        v_issued_count = 0;
     }
     if (threadIdx.x < 4) cx.rflag[threadIdx.x] = -1;
+    // The layers of one forward pass see the same per-scene counts, so the work split is made once
+    // per pass (a launch of this kernel with split_only set) and kept in the memo, with the counts it
+    // was computed from.  The memo's loads and those of the counts are all issued before the first
+    // use, so that they share one trip to memory; when they may be read ahead of the dependency wait
+    // they are issued right here, and the trip hides behind the set-up.
+    constexpr int MEMO_MAGIC = 0x5D170000 | (W_PREFIX << 12) | (W_MASKED << 8) | W_PAIR;
+    const int32_t* mrd = (p.split_memo && !split_only) ? p.split_memo : nullptr;
+    int4 mh0 = make_int4(0, 0, 0, 0), mh1 = mh0, mh2 = mh0, me = mh0;
+    int m_na = -1, m_nt = -1, m_prev = 0;
+    int na[4], nt[4];
+    auto issue_loads = [&]() {
+        if (mrd) {
+            mh0 = __ldcg(reinterpret_cast<const int4*>(mrd));
+            mh1 = __ldcg(reinterpret_cast<const int4*>(mrd) + 1);
+            mh2 = __ldcg(reinterpret_cast<const int4*>(mrd) + 2);
+            me = __ldcg(reinterpret_cast<const int4*>(mrd + FDC_MEMO_ENTRIES) + blockIdx.x);
+            if ((int)threadIdx.x < p.batch) {
+                m_na = __ldcg(mrd + 16 + threadIdx.x);
+                m_nt = __ldcg(mrd + 16 + FDC_MEMO_BATCH + threadIdx.x);
+            }
+            if ((int)threadIdx.x <= p.batch) m_prev = __ldcg(mrd + 16 + 2 * FDC_MEMO_BATCH + threadIdx.x);
+        }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int i = threadIdx.x + j * THREADS;
+            na[j] = i < p.batch ? p.n_active[i] : 0;
+            nt[j] = i < p.batch ? p.ntiles[i] : 0;
+        }
+    };
+    if (p.early) issue_loads();
     // ---- set-up that needs no global memory: barriers, TMEM
     if (threadIdx.x == 0) {
         for (int i = 0; i < MAXST; ++i) {
@@ -1294,7 +1299,6 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, con
             mbar_init(cx.k_empty + 8 * i, 1);
             mbar_init(cx.v_full + 8 * i, 1);
             mbar_init(cx.v_empty + 8 * i, 1);
-            mbar_init(cx.v_clean + 8 * i, 1);
         }
         for (int i = 0; i < 4; ++i) {
             mbar_init(cx.s_full + 8 * i, 1);
@@ -1310,7 +1314,7 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, con
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         fence_async_smem();
     }
-    if (warp == W_QK) {
+    if (warp == W_QK && !split_only) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_holder)), "r"(TMEM_COLS)
                      : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -1318,43 +1322,24 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, con
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    const uint32_t tmem = *reinterpret_cast<volatile uint32_t*>(tmem_holder);
+    const uint32_t tmem = split_only ? 0u : *reinterpret_cast<volatile uint32_t*>(tmem_holder);
     cx.tmem = tmem;
     // Programmatic dependent launch: this grid may have been scheduled while the kernel before it in
-    // the stream was still running.  Nothing of global memory is touched before that kernel has
-    // completed; the kernel after this one may be scheduled early in the same way.
-    asm volatile("griddepcontrol.wait;" ::: "memory");
+    // the stream was still running, and the kernel after this one may be scheduled early in the same
+    // way.  Ordinarily nothing of global memory is touched before the kernel ahead has completed, and
+    // only then is the next one let in.  With p.early the host vouches that the pass tables (counts,
+    // tile lists, bitmaps), the work split and the prefix rows of the cache were complete before the
+    // kernel ahead even began: then the work split is looked up and the first K/V stages of the prefix
+    // are requested right away, while that kernel's last blocks are still running, and only what it
+    // may have written (queries, the pass's new K/V rows, the rows beyond the prefix) waits for it.
+    // Every thread passes the wait before the block ends, so grids complete in stream order.
+    if (!p.early) asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    if (!p.early) issue_loads();
     bool active = true;                       // this CTA has units (uniform over the CTA)
     long long lo = 0, hi = 0;
-    // The layers of one forward pass see the same per-scene counts, so the previous launch on this
-    // plan has left its work split in the memo, with the counts it was computed from.  Its loads
-    // are issued first; they are in flight together with those of the counts.
-    constexpr int MEMO_MAGIC = 0x5D170000 | (W_MASKED << 8) | W_PAIR;
-    const int32_t* mrd = p.split_memo ? p.split_memo + ((p.seq - 1u) & 1u) * FDC_MEMO_INTS : nullptr;
-    int4 mh0 = make_int4(0, 0, 0, 0), mh1 = mh0, mh2 = mh0, me = mh0;
-    int m_na = -1, m_nt = -1, m_prev = 0;
-    if (mrd) {
-        mh0 = __ldcg(reinterpret_cast<const int4*>(mrd));
-        mh1 = __ldcg(reinterpret_cast<const int4*>(mrd) + 1);
-        mh2 = __ldcg(reinterpret_cast<const int4*>(mrd) + 2);
-        me = __ldcg(reinterpret_cast<const int4*>(mrd + FDC_MEMO_ENTRIES) + blockIdx.x);
-        if ((int)threadIdx.x < p.batch) {
-            m_na = __ldcg(mrd + 16 + threadIdx.x);
-            m_nt = __ldcg(mrd + 16 + FDC_MEMO_BATCH + threadIdx.x);
-        }
-        if ((int)threadIdx.x <= p.batch) m_prev = __ldcg(mrd + 16 + 2 * FDC_MEMO_BATCH + threadIdx.x);
-    }
-    // the counts: every load is issued before the first use, so that all of them (and the memo's)
-    // share one trip to memory; the raw tile counts wait in prev[] for the scan
+    // the raw tile counts wait in prev[] for the scan
     {
-        int na[4], nt[4];
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const int i = threadIdx.x + j * THREADS;
-            na[j] = i < p.batch ? p.n_active[i] : 0;
-            nt[j] = i < p.batch ? p.ntiles[i] : 0;
-        }
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
             const int i = threadIdx.x + j * THREADS;
@@ -1378,7 +1363,7 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, con
     cx.npre = p.P / TILE;
     bool hit = false;
     if (mrd) {
-        int same = mh0.x == MEMO_MAGIC && mh0.y == (int)(p.seq - 1u) && mh0.z == p.hkv && mh0.w == p.n_cta && mh1.x == p.P && mh1.y == p.batch;
+        int same = mh0.x == MEMO_MAGIC && mh0.y == (int)p.seq && mh0.z == p.hkv && mh0.w == p.n_cta && mh1.x == p.P && mh1.y == p.batch;
         if ((int)threadIdx.x < p.batch) same = same && m_na == cx.nact[threadIdx.x] && m_nt == cx.pre[threadIdx.x + 1] - cx.pre[threadIdx.x];
         hit = __syncthreads_and(same) != 0;
     }
@@ -1484,7 +1469,7 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, con
                 hi = lo + (j1 - j0);
             }
         } else {
-            const long long want = (U + MIN_UNITS - 1) / MIN_UNITS;      // small problems use fewer CTAs
+            const long long want = (U + MIN_TILES - 1) / MIN_TILES;      // small problems use fewer CTAs
             if (want < cx.n_cta) cx.n_cta = (int)want;
             cx.vtot = (long long)cx.prev[p.batch] * p.hkv;
             lo = unit_of_virt(p, cx, cta_first_unit(blockIdx.x, cx.vtot, cx.n_cta));
@@ -1496,9 +1481,9 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, con
         hi = cta_first_unit(blockIdx.x + 1, U, cx.n_cta);
     }
     if (lo >= hi || (int)blockIdx.x >= cx.n_cta) active = false;
-    if (p.split_memo) {
-        // leave the split to the next launch (plain stores, nobody waits for them)
-        int32_t* mwr = p.split_memo + (p.seq & 1u) * FDC_MEMO_INTS;
+    if (split_only) {
+        // this launch only computes the split and leaves it to the attention launches of the pass
+        int32_t* mwr = p.split_memo;
         if (threadIdx.x == 0)
             reinterpret_cast<int4*>(mwr + FDC_MEMO_ENTRIES)[blockIdx.x] =
                 active ? make_int4((int)(uint32_t)lo, (int)(lo >> 32), (int)(uint32_t)hi, (int)(hi >> 32)) : make_int4(0, 0, 0, 0);
@@ -1516,11 +1501,16 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, con
         }
     }
 
+    if (split_only) active = false;
+    // Two roles run ahead of the dependency wait (with p.early): the TMA producer, which takes the wait
+    // itself once nothing more of the prefix can be requested, and the softmax warps, which first stage
+    // the first pair's bitmaps.
+    if (p.early && !(active && (warp == W_PROD || warp < NSOFT))) asm volatile("griddepcontrol.wait;" ::: "memory");
     if (!active) {
     } else if (warp == W_PROD) {
         producer_loop(p, cx, &tm_k, &tm_v, lo, hi, lane);
-    } else if (warp == W_CLEAN) {
-        clean_loop(p, cx, lo, hi, lane);
+    } else if (warp == W_AUX) {
+        aux_loop(p, cx, lo, hi, lane);
     } else if (warp == W_PV) {
         pv_loop(p, cx, lo, hi, lane);
     } else if (warp == W_QK) {
@@ -1528,13 +1518,23 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, con
     } else {
         int s = 0;
         uint32_t g = 0, seg = 0;
+        int vst = 0;                              // V ring stage and phase of round g
+        uint32_t vph = 0;
         long long u = lo;
         bool dead = false;                        // a bounded wait ran out somewhere in the CTA
         int prefetched = 0;                       // the segment's queries and bitmaps are already on their way
+        if (p.early) {
+            // ahead of the dependency wait: the first pair's bitmaps; its queries follow right after the wait
+            int s0 = 0;
+            const Segment sg = decode_segment(lo, hi, cx.pre, p.hkv, s0);
+            stage_first_pair_early(reinterpret_cast<const uint4*>(p.q), p.mask, p.max_active, p.W, p.hq, p.group, sg.s, sg.g,
+                                   cx.nact[sg.s] * p.group, cx.qs, cx.q_panel, cx.mstaged ? cx.smask : nullptr);
+            prefetched = 1;
+        }
         while (u < hi) {
             const Segment sg = decode_segment(u, hi, cx.pre, p.hkv, s);
             const int M = cx.nact[sg.s] * p.group;
-            softmax_segment(p, cx, sg, (M <= 32 ? 32 : (M <= 64 ? 64 : 128)) / NPART, seg, hi, prefetched, g, dead, warp, lane);
+            softmax_segment(p, cx, sg, (M <= 32 ? 32 : (M <= 64 ? 64 : 128)) / NPART, seg, hi, prefetched, g, vst, vph, dead, warp, lane);
             ++seg;
             u = sg.next_u;
         }
@@ -1542,7 +1542,7 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, con
     // ---- teardown: everybody is done with TMEM before it is freed
     tc_fence_before();
     __syncthreads();
-    if (warp == W_QK) {
+    if (warp == W_QK && !split_only) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(TMEM_COLS) : "memory");
     }
@@ -1553,8 +1553,9 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, con
 namespace fdc {
 
 // bf16, head_dim 128, at most 128 query rows per (scene, KV head); FDC_ERR_SHAPE otherwise (the
-// caller then takes another kernel).
-int launch_attn_tc(const AttnParams& p, int head_dim, cudaStream_t st)
+// caller then takes another kernel).  split_only: the launch only computes the work split of the
+// pass into p.split_memo (an ordinary launch; no rings, no TMEM).
+static int launch_tc(const AttnParams& p, int head_dim, cudaStream_t st, int split_only)
 {
     if (head_dim != D || p.mmax > 128) return FDC_ERR_SHAPE;
     const int np_max = p.mmax <= 32 ? 32 : (p.mmax <= 64 ? 64 : 128);
@@ -1565,6 +1566,7 @@ int launch_attn_tc(const AttnParams& p, int head_dim, cudaStream_t st)
     int stages = (int)((227 * 1024 - 256 - fixed) / STAGE);
     if (stages > 2 * MAXST) stages = 2 * MAXST;
     if (stages < 4) return FDC_ERR_SHAPE;
+    if (split_only) stages = 0;
     const int nk = stages / 2, nv = stages - nk;
     const size_t smem = fixed + (size_t)stages * STAGE;
     alignas(64) CUtensorMap tk, tv;
@@ -1572,11 +1574,17 @@ int launch_attn_tc(const AttnParams& p, int head_dim, cudaStream_t st)
     if (rc) return rc;
     rc = get_kv_tensor_map(p.v, p, D, TILE, &tv);
     if (rc) return rc;
-    static size_t attr_smem = 0;
-    if (smem > attr_smem) {
+    // the attribute is kept per device by the runtime
+    static size_t attr_smem[64] = {};
+    int dev = 0;
+    {
+        cudaError_t e = cudaGetDevice(&dev);
+        if (e != cudaSuccess) return set_cuda_error(e);
+    }
+    if (dev < 0 || dev >= 64 || smem > attr_smem[dev]) {
         cudaError_t e = cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return set_cuda_error(e);
-        attr_smem = smem;
+        if (dev >= 0 && dev < 64) attr_smem[dev] = smem;
     }
     {
         cudaLaunchConfig_t cfg = {};
@@ -1588,13 +1596,16 @@ int launch_attn_tc(const AttnParams& p, int head_dim, cudaStream_t st)
         at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
         at[0].val.programmaticStreamSerializationAllowed = 1;
         cfg.attrs = at;
-        cfg.numAttrs = 1;
-        cudaError_t e = cudaLaunchKernelEx(&cfg, attn_tc_kernel, p, tk, tv, nk, nv, np_max, npb);
+        cfg.numAttrs = split_only ? 0 : 1;
+        cudaError_t e = cudaLaunchKernelEx(&cfg, attn_tc_kernel, p, tk, tv, nk, nv, np_max, npb, split_only);
         if (e != cudaSuccess) return set_cuda_error(e);
     }
     note_launch();
     cudaError_t e = cudaGetLastError();
     return e == cudaSuccess ? FDC_OK : set_cuda_error(e);
 }
+
+int launch_attn_tc(const AttnParams& p, int head_dim, cudaStream_t st) { return launch_tc(p, head_dim, st, 0); }
+int launch_attn_tc_split(const AttnParams& p, int head_dim, cudaStream_t st) { return launch_tc(p, head_dim, st, 1); }
 
 }  // namespace fdc

@@ -7,11 +7,12 @@
 #include "fdc.h"
 
 #define FDC_PAIR_COUNTERS 65536
-// Work-split memo of the tcgen05 attention kernel: the layers of one forward pass see the same
-// per-scene counts, so the split of one launch is kept (with the counts it was computed from) and
-// the next launch only checks that the counts are unchanged.  Layout of a slot, in int32:
-// [0..15] header, [16..) n_active[FDC_MEMO_BATCH], tiles[FDC_MEMO_BATCH], prev[FDC_MEMO_BATCH + 1],
-// [FDC_MEMO_ENTRIES..) first and last unit of each CTA (2 x int64).
+// Work split of the tcgen05 attention kernel: the layers of one forward pass see the same
+// per-scene counts, so the split is computed once per pass (by a launch of the kernel that does
+// nothing else, before the pass's first attention launch) and kept here with the counts it was
+// computed from; the attention launches only check that the counts are unchanged.  Layout, in
+// int32: [0..15] header, [16..) n_active[FDC_MEMO_BATCH], tiles[FDC_MEMO_BATCH],
+// prev[FDC_MEMO_BATCH + 1], [FDC_MEMO_ENTRIES..) first and last unit of each CTA (2 x int64).
 #define FDC_MEMO_BATCH 256
 #define FDC_MEMO_CTAS 256
 #define FDC_MEMO_ENTRIES 800
@@ -58,14 +59,29 @@ struct fdc_pending_append {
     void*          stream;
 };
 
+// Everything the work split of the tcgen05 attention kernel depends on (host side).
+struct fdc_split_key {
+    uint32_t       tables_gen;
+    const int32_t* d_n_active;
+    const int32_t* d_ntiles;
+    int32_t        batch, hkv, n_cta, P;
+    void*          stream;
+    int            valid;
+};
+
 struct fdc_plan {
     fdc::PlanDev  h;                 // host copy
     fdc::PlanDev* d;                 // device copy
     int32_t*      d_status;          // sticky FDC_DEV_* bits
     int32_t*      d_ticket;          // [2] scratch of the frontier kernel's cross-block reduction
     int32_t*      d_pair_cnt;        // [FDC_PAIR_COUNTERS] arrivals per (scene, KV head) of the fused combine (zero between calls)
-    int32_t*      d_split_memo;      // [2][FDC_MEMO_INTS] work split of the last attention launch and the counts it was made from
-    uint32_t      attn_seq;          // attention launches on this plan so far (selects the memo slot)
+    int32_t*      d_split_memo;      // [FDC_MEMO_INTS] work split of the current pass and the counts it was made from
+    uint32_t      tables_gen;        // bumped by every call that rewrites the pass tables (state_init, frontier, build_masks)
+    uint32_t      split_gen;         // number of the last split launch (stored in the memo's header)
+    fdc_split_key split_key;         // what the memo was computed for
+    uint32_t      attn_gen;          // tables_gen at the last attention launch of the tcgen05 kernel
+    void*         attn_stream;       // and its stream
+    int           attn_gen_valid;
     int           fuse_append;       // fdc_set_fused_append
     fdc_pending_append pend;         // recorded append waiting for its attention call
     int           device;
@@ -96,8 +112,10 @@ struct AttnParams {
     float           scale_log2;      // softmax scale * log2(e)
     int32_t*        status;          // sticky FDC_DEV_* bits
     int32_t*        pair_cnt;        // per (scene, KV head) arrival counters: the split kernel also combines (nullptr: it does not)
-    int32_t*        split_memo;      // [2][FDC_MEMO_INTS] (nullptr: the work split is always computed)
-    uint32_t        seq;             // number of this launch on the plan
+    int32_t*        split_memo;      // [FDC_MEMO_INTS] (nullptr: the work split is always computed)
+    uint32_t        seq;             // number of the split launch the memo must come from
+    int32_t         early;           // the pass tables, the memo and the prefix rows were complete before the kernel
+                                     // preceding this one in the stream began: they may be read ahead of the dependency wait
     const int32_t*  app_row;         // fused append: [batch][max_active] cache row of each branch's new K/V vector (nullptr: none)
     const void*     app_k;           // [batch][max_active][hkv][D]
     const void*     app_v;
@@ -110,13 +128,14 @@ int  set_cuda_error(cudaError_t e);                  // records the message, ret
 int launch_attn_ref(const AttnParams& p, int dtype, int head_dim, cudaStream_t st);
 int launch_attn_mma(const AttnParams& p, int head_dim, cudaStream_t st);
 int launch_attn_tc(const AttnParams& p, int head_dim, cudaStream_t st);
+int launch_attn_tc_split(const AttnParams& p, int head_dim, cudaStream_t st);   // computes the work split only (into p.split_memo)
 int launch_attn_combine(const AttnParams& p, int dtype, int head_dim, cudaStream_t st);
 void prof_destroy(fdc_plan* plan);
 int  check_kv_desc(const fdc_plan* plan, const fdc_kv_desc* kv, int32_t layer);
 bool takes_tc_kernel(const fdc_plan* plan, const fdc_kv_desc* kv);   // fdc_decode_attn would run the tcgen05 kernel with the combine fused in
-int  launch_kv_append(const fdc_plan* plan, const fdc_kv_desc* kv, int32_t layer, const int32_t* d_n_active, const int32_t* d_kv_row,
+int  launch_kv_append(fdc_plan* plan, const fdc_kv_desc* kv, int32_t layer, const int32_t* d_n_active, const int32_t* d_kv_row,
                       const void* d_k_new, const void* d_v_new, void* stream);
-int  flush_pending_append(const fdc_plan* plan);     // launches a recorded append on its own (no-op when there is none)
+int  flush_pending_append(fdc_plan* plan);     // launches a recorded append on its own (no-op when there is none)
 
 // ----------------------------------------------------------------------------------
 // device helpers

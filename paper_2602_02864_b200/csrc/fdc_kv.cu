@@ -92,7 +92,7 @@ int check_kv_desc(const fdc_plan* p, const fdc_kv_desc* kv, int32_t layer)
 
 namespace fdc {
 
-int launch_kv_append(const fdc_plan* p, const fdc_kv_desc* kv, int32_t layer, const int32_t* d_n_active, const int32_t* d_kv_row,
+int launch_kv_append(fdc_plan* p, const fdc_kv_desc* kv, int32_t layer, const int32_t* d_n_active, const int32_t* d_kv_row,
                      const void* d_k_new, const void* d_v_new, void* stream)
 {
     const int es = kv->dtype == FDC_F32 ? 4 : 2;
@@ -123,9 +123,8 @@ int launch_kv_append(const fdc_plan* p, const fdc_kv_desc* kv, int32_t layer, co
     return FDC_OK;
 }
 
-int flush_pending_append(const fdc_plan* plan)
+int flush_pending_append(fdc_plan* p)
 {
-    fdc_plan* p = const_cast<fdc_plan*>(plan);
     if (!p || !p->pend.valid) return FDC_OK;
     p->pend.valid = 0;
     return launch_kv_append(p, &p->pend.kv, p->pend.layer, p->pend.d_n_active, p->pend.d_kv_row, p->pend.d_k_new, p->pend.d_v_new,
@@ -134,7 +133,7 @@ int flush_pending_append(const fdc_plan* plan)
 
 }  // namespace fdc
 
-extern "C" int fdc_kv_append(const fdc_plan* p, const fdc_kv_desc* kv, int32_t layer, const int32_t* d_n_active,
+extern "C" int fdc_kv_append(fdc_plan* p, const fdc_kv_desc* kv, int32_t layer, const int32_t* d_n_active,
                              const int32_t* d_kv_row, const void* d_k_new, const void* d_v_new, void* stream)
 {
     int rc = check_kv_desc(p, kv, layer);

@@ -230,7 +230,7 @@ __global__ void __launch_bounds__(256) build_masks_kernel(const PlanDev* __restr
 
 extern "C" {
 
-int fdc_state_init(const fdc_plan* p, int32_t batch, const int32_t* d_len, void* d_state, void* stream)
+int fdc_state_init(fdc_plan* p, int32_t batch, const int32_t* d_len, void* d_state, void* stream)
 {
     if (!p || !d_state) return FDC_ERR_NULL;
     if (batch < 1 || batch > FDC_MAX_BATCH) return FDC_ERR_RANGE;
@@ -239,6 +239,7 @@ int fdc_state_init(const fdc_plan* p, int32_t batch, const int32_t* d_len, void*
         if (rcf) return rcf;
     }
     const int warps = 4;
+    ++p->tables_gen;                       // the pass tables change: work splits made from them are stale
     state_init_kernel<<<(batch + warps - 1) / warps, warps * 32, 0, (cudaStream_t)stream>>>(
         p->d, batch, d_len, (SceneState*)d_state, p->d_status);
     note_launch();
@@ -246,7 +247,7 @@ int fdc_state_init(const fdc_plan* p, int32_t batch, const int32_t* d_len, void*
     return FDC_OK;
 }
 
-int fdc_frontier(const fdc_plan* p, int32_t batch, void* d_state, const uint8_t* d_finish, int32_t* d_n_active,
+int fdc_frontier(fdc_plan* p, int32_t batch, void* d_state, const uint8_t* d_finish, int32_t* d_n_active,
                  int32_t* d_node, int32_t* d_tok_idx, int32_t* d_kv_row, int32_t* d_pos_id,
                  int32_t* d_all_done, void* stream)
 {
@@ -258,6 +259,7 @@ int fdc_frontier(const fdc_plan* p, int32_t batch, void* d_state, const uint8_t*
         if (rcf) return rcf;
     }
     const int warps = batch < 8 ? batch : 8;
+    ++p->tables_gen;                       // the pass tables change: work splits made from them are stale
     frontier_kernel<<<(batch + warps - 1) / warps, warps * 32, 0, (cudaStream_t)stream>>>(
         p->d, batch, (SceneState*)d_state, d_finish, d_n_active, d_node, d_tok_idx, d_kv_row, d_pos_id,
         d_all_done, p->d_status, p->d_ticket);
@@ -266,7 +268,7 @@ int fdc_frontier(const fdc_plan* p, int32_t batch, void* d_state, const uint8_t*
     return FDC_OK;
 }
 
-int fdc_build_masks(const fdc_plan* p, int32_t batch, const void* d_state, uint64_t* d_mask, uint64_t* d_umask,
+int fdc_build_masks(fdc_plan* p, int32_t batch, const void* d_state, uint64_t* d_mask, uint64_t* d_umask,
                     int32_t* d_tiles, int32_t* d_ntiles, void* stream)
 {
     if (!p || !d_state || !d_mask || !d_umask || !d_tiles || !d_ntiles) return FDC_ERR_NULL;
@@ -275,6 +277,7 @@ int fdc_build_masks(const fdc_plan* p, int32_t batch, const void* d_state, uint6
         int rcf = flush_pending_append(p);
         if (rcf) return rcf;
     }
+    ++p->tables_gen;                       // the pass tables change: work splits made from them are stale
     build_masks_kernel<<<batch, 256, p->h.W * sizeof(uint64_t), (cudaStream_t)stream>>>(
         p->d, (const SceneState*)d_state, d_mask, d_umask, d_tiles, d_ntiles);
     note_launch();

@@ -198,10 +198,10 @@ def test_softmax_reference_is_raised_when_scores_jump(monkeypatch):
 
 
 def test_work_split_of_the_previous_call_is_reused_only_for_the_same_counts():
-    """The attention kernel keeps its work split in the plan for the next call and reuses it
-    when n_active and ntiles are unchanged.  A repeated call must give the same bits; a call
-    with other counts (one scene switched off) must not use the stale split; and going back
-    to the first counts must reproduce the first result."""
+    """The work split of a pass is computed once (before its first attention call) and kept in
+    the plan.  A repeated call must give the same bits; a call with other counts (one scene
+    switched off, in other arrays or in the same ones) must not use the stale split; and going
+    back to the first counts must reproduce the first result."""
     from paper_2602_02864_b200 import fdc
     from harness import alloc_cache, write_prefix, BF16_MAX_ABS, f32
     w = wl.cfg2_batched(layers=1, batch=4)
@@ -237,6 +237,16 @@ def test_work_split_of_the_previous_call_is_reused_only_for_the_same_counts():
         assert np.abs(f32(other[s, :A]) - f32(first[s, :A])).max() <= BF16_MAX_ABS
     back = attend(sess.n_active, sess.ntiles)
     assert torch.equal(first, back)
+    # the same arrays with other contents (behind the library's back): the kernel itself notices that
+    # the kept split was made from other counts and makes its own
+    keep = (sess.n_active.clone(), sess.ntiles.clone())
+    sess.n_active[1] = 0
+    sess.ntiles[1] = 0
+    inplace = attend(sess.n_active, sess.ntiles)
+    assert torch.equal(inplace, other)
+    sess.n_active.copy_(keep[0])
+    sess.ntiles.copy_(keep[1])
+    assert torch.equal(first, attend(sess.n_active, sess.ntiles))
     assert sess.status() == 0
     sess.close()
 
