@@ -54,6 +54,20 @@ constexpr int PANEL = RROWS * 128;           // 128 rows x 128 bytes (64 bf16 co
 constexpr int STAGE = (D / 64) * PANEL;      // one K (or V) stage: 128 rows x head_dim
 constexpr int MAXST = 4;                     // stages per ring at most
 constexpr float RAISE_LOG2 = 16.f;
+// Event trace for development builds (-DFDC_TRACE=<CTA>): clock64 stamps of one CTA, per round and
+// per segment, read back with fdc_tr_read.  Compiled out otherwise.
+#ifdef FDC_TRACE
+__device__ long long g_tr[64 * 16];
+__device__ long long g_ts[80];
+#define FDC_TRC ((int)blockIdx.x == FDC_TRACE)
+#define FDC_TR(g, e) do { if (FDC_TRC && (g) < 64) g_tr[(g) * 16 + (e)] = clock64(); } while (0)
+#define FDC_TS(e) do { if (FDC_TRC) g_ts[e] = clock64(); } while (0)
+#define FDC_TSS(e) do { if (FDC_TRC && seg < 4) g_ts[16 + seg * 16 + (e)] = clock64(); } while (0)
+#else
+#define FDC_TR(g, e) do { } while (0)
+#define FDC_TS(e) do { } while (0)
+#define FDC_TSS(e) do { } while (0)
+#endif
 constexpr float UNSET = 1.0e30f;             // -reference of a column that has seen nothing yet
 #ifndef FDC_W_PREFIX
 #define FDC_W_PREFIX 4
@@ -375,10 +389,12 @@ __device__ __forceinline__ void producer_loop(const AttnParams& p, const Ctx& cx
         rk = __shfl_sync(0xffffffffu, rk, 0);
         rv = __shfl_sync(0xffffffffu, rv, 0);
         if (rk) {
+            if (lane == 0) FDC_TR(ck.g, 12);
             cursor_issue(ck, tm_k, cx.kring, cx.k_full, pol, lane);
             cursor_next(ck, p, cx, hi, cx.nk, lane);
         }
         if (rv) {
+            if (lane == 0) FDC_TR(cv.g, 13);
             cursor_issue(cv, tm_v, cx.vring, cx.v_full, pol, lane);
             cursor_next(cv, p, cx, hi, cx.nv, lane);
         }
@@ -442,9 +458,11 @@ __device__ __forceinline__ void qk_loop(const AttnParams& p, const Ctx& cx, long
             bool good = mbar_wait(cx.q_ready, seg & 1, cx.abortp, p.status);
             for (int t = 0; t < nr && good; ++t, ++g) {
                 good = mbar_wait(cx.k_full + 8 * st, kph, cx.abortp, p.status);
+                FDC_TR(g, 6);
                 const uint32_t sb = g & (cx.ns - 1);                  // score buffer of the round
                 if (good && g >= (uint32_t)cx.ns) good = mbar_wait(cx.s_free + 8 * sb, ((g / cx.ns) - 1) & 1, cx.abortp, p.status);
                 if (!good) break;
+                FDC_TR(g, 7);
                 tc_fence_after();
                 const uint32_t kd = k_lo0 + (uint32_t)((st * STAGE) >> 4);
                 const uint32_t d = cx.tmem + sb * cx.s_stride;
@@ -454,6 +472,7 @@ __device__ __forceinline__ void qk_loop(const AttnParams& p, const Ctx& cx, long
                           idesc_qk, ks > 0);
                 umma_commit(cx.k_empty + 8 * st);
                 umma_commit(cx.s_full + 8 * sb);
+                FDC_TR(g, 8);
                 if (++st == cx.nk) {
                     st = 0;
                     kph ^= 1;
@@ -578,9 +597,11 @@ __device__ __forceinline__ void pv_loop(const AttnParams& p, const Ctx& cx, long
             bool good = true;
             for (int t = 0; 2 * t < ntile && good; ++t, ++g) {
                 good = mbar_wait(cx.v_full + 8 * st, vph, cx.abortp, p.status);
+                FDC_TR(g, 9);
                 if (good) good = mbar_wait(cx.p_full + 8 * (g & 1), (g >> 1) & 1, cx.abortp, p.status);
                 if (good && t == 0 && seg > 0) good = mbar_wait(cx.o_free, (seg - 1) & 1, cx.abortp, p.status);
                 if (!good) break;
+                FDC_TR(g, 10);
                 const uint32_t steps = (uint32_t)cx.v_steps[(g & 1) * 2] | ((uint32_t)cx.v_steps[(g & 1) * 2 + 1] << 4);
                 tc_fence_after();
                 const uint32_t vd = v_lo0 + (uint32_t)((st * STAGE) >> 4);
@@ -601,6 +622,7 @@ __device__ __forceinline__ void pv_loop(const AttnParams& p, const Ctx& cx, long
                 }
                 umma_commit(cx.v_empty + 8 * st);
                 umma_commit(cx.pv_done + 8 * (g & 1));
+                FDC_TR(g, 11);
                 if (++st == cx.nv) {
                     st = 0;
                     vph ^= 1;
@@ -886,11 +908,14 @@ __device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& 
         if (!mbar_wait_slow(bar, parity, cx.abortp, p.status)) dead = true;
         dead = __any_sync(0xffffffffu, dead);
     };
+    if (tid == 0 && seg == 0) FDC_TS(5);
+    if (tid == 0) FDC_TSS(0);
     // ---- Q^T (B operand of S^T = K Q^T): row n = query row, K-major, 128B swizzle, rows >= M zero
+    const bool published = prefetched == 2;       // Q^T, the bitmaps and their OR were completed and announced at the end of the previous segment
     {
         if (prefetched) {
             // queries and bitmaps were copied asynchronously during the previous segment's last round
-            cp_async_wait_all();
+            if (!published) cp_async_wait_all();
             prefetched = 0;
         } else {
             // all global reads first (one latency), then the stores
@@ -926,7 +951,7 @@ __device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& 
                 if (idx < nw) cx.smask[(seg & 1) * MBUF + idx] = mv[i];
             }
         }
-        if (cx.mstaged && p.W <= UW) {
+        if (cx.mstaged && p.W <= UW && !published) {
             // OR of the scene's bitmaps: the rows that some branch may see (the others are cleared in V)
             soft_sync();                              // everybody's share of the bitmaps is in place
             if (tid < p.W) {
@@ -944,10 +969,14 @@ __device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& 
             for (int ch = 0; ch < nch; ++ch) tmem_st<8>(l_addr + ch * 8, z);      // column sums start at 0
             tmem_wait_st();
         }
-        fence_async_smem();
-        __syncwarp();
-        if (!dead && lane == 0) mbar_arrive(cx.q_ready);
+        if (!published) {
+            fence_async_smem();
+            __syncwarp();
+            if (!dead && lane == 0) mbar_arrive(cx.q_ready);
+        }
         soft_sync();
+        if (tid == 0 && seg == 0) FDC_TS(6);
+        if (tid == 0) FDC_TSS(1);
     }
 
     const int ntile = sg.j1 - sg.j0;
@@ -958,6 +987,7 @@ __device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& 
         for (int k = 0; k < jn; k += 2, ++g, ++t) {
             const int nt = jn - k < 2 ? 1 : 2;
             const uint32_t b = g & 1;
+            if (tid == 0) FDC_TR(g, 0);
             const int ti = q4 >> 1;                                   // which tile of the round this warp's rows are in
             const int tile = __shfl_sync(0xffffffffu, my_tile, (k + ti) & 31);
             const bool live = ti < nt && !dead;                       // rows 64..127 of a one-tile round hold nothing
@@ -967,7 +997,8 @@ __device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& 
             const uint32_t sb = g & (cx.ns - 1);                      // score buffer of the round
             wait_u(cx.s_full + 8 * sb, (g / cx.ns) & 1);
             tc_fence_after();
-            if (jb + k + 2 >= ntile && sg.next_u < hi && !dead) {
+            if (tid == 0) FDC_TR(g, 1);
+            if (jb + k + 2 >= ntile && sg.next_u < hi) {
                 // last round: every S^T = K Q^T of this segment has completed, so Q^T may be overwritten.
                 // The next segment's queries (and its scene's bitmaps, into the other buffer) are copied
                 // asynchronously; the latency hides behind this round, the drain and the partial write.
@@ -980,6 +1011,7 @@ __device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& 
             // warp has also finished round g - 2, so what that round left in rflag is the same for all.
             if (cx.npb == 2) wait_u(cx.pv_done + 8 * b, ((g >> 1) & 1) ^ 1);
             else if (g > 0) wait_u(cx.pv_done + 8 * ((g - 1) & 1), ((g - 1) >> 1) & 1);
+            if (tid == 0) FDC_TR(g, 2);
             const uint32_t s_addr = cx.tmem + lane_base + sb * cx.s_stride + col0;
             // References are set in the first round of a segment.  Later a score more than 2^16 above its
             // reference only leaves a note (no barrier in the common path): p stays far from overflow, and
@@ -1020,6 +1052,7 @@ __device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& 
                 ra.dead = dead;
                 dead = raise_references(ra) != 0;
             }
+            if (tid == 0) FDC_TR(g, 3);
             if (live) {
                 unsigned char* prow = cx.ps + (b & (cx.npb - 1)) * cx.p_buf + krow * 128;
                 float emax = 0.f;
@@ -1065,6 +1098,7 @@ __device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& 
                     if (!(emax < 1.0e30f)) atomicOr(p.status, FDC_DEV_SCORE_RANGE);     // beyond 2^100 (or inf / nan)
                 }
             }
+            if (tid == 0) FDC_TR(g, 4);
             // ---- this round's V stage.  Beyond the prefix, rows that no branch of the scene may see can hold
             // anything (NaN, Inf: slots that were never written), and although their P^T entries are
             // exactly 0, 0 * NaN must not reach the accumulator.  The multiplication runs in steps of 16
@@ -1106,12 +1140,36 @@ __device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& 
                 mbar_arrive(cx.s_free + 8 * sb);                       // the scores have been read: K Q^T may reuse the buffer
                 mbar_arrive(cx.p_full + 8 * b);
             }
+            if (tid == 0) FDC_TR(g, 5);
         }
+    }
+    if (tid == 0) { FDC_TS(7); FDC_TSS(2); }
+    if (prefetched == 1) {
+        // The next pair's queries are announced before this pair is finished off, so that its K Q^T runs
+        // on (into the score buffers) while the last multiplications drain and the result is written.
+        cp_async_wait_all();
+        if (cx.mstaged && p.W <= UW) {
+            soft_sync();
+            int s2 = sg.s;
+            const Segment nx = decode_segment(sg.next_u, hi, cx.pre, p.hkv, s2);
+            if (tid < p.W) {
+                const uint64_t* mb = cx.smask + ((seg + 1) & 1) * MBUF + tid;
+                uint64_t un = 0ull;
+                const int A2 = cx.nact[nx.s];
+                for (int b = 0; b < A2; ++b) un |= mb[(size_t)b * p.W];
+                cx.sunion[((seg + 1) & 1) * UW + tid] = un;
+            }
+        }
+        fence_async_smem();
+        __syncwarp();
+        if (!dead && lane == 0) mbar_arrive(cx.q_ready);
+        prefetched = 2;
     }
     // ---- end of segment: the accumulator is final once the last PV has completed
     const uint32_t last = g - 1;
     wait_u(cx.pv_done + 8 * (last & 1), (last >> 1) & 1);
     tc_fence_after();
+    if (tid == 0) { FDC_TS(8); FDC_TSS(3); }
     // column sums over the warp's 32 rows by transpose-reduce: lane i < 8 ends up with column i's sum
 #pragma unroll 1
     for (int ch = 0; ch < nch; ++ch) {
@@ -1140,6 +1198,7 @@ __device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& 
     const int pair = sg.s * p.hkv + sg.g;
     const int slot = blockIdx.x + pair;
     const bool whole = sg.j0 == 0 && sg.j1 == sg.nt;       // this CTA saw every tile of the pair
+    if (tid == 0) FDC_TSS(4);
     if (p.pair_cnt && whole) {
         // no other partial exists: normalise and write the output directly
         if (tid < np) cx.alpha[tid] = 1.f / ((cx.lred[tid] + cx.lred[128 + tid]) + (cx.lred[256 + tid] + cx.lred[384 + tid]));
@@ -1184,6 +1243,7 @@ __device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& 
                     if (col0 + ch * 8 + i < M) wo[(size_t)(col0 + ch * 8 + i) * D] = __uint_as_float(ov[i]);
             }
         }
+        if (tid == 0) FDC_TSS(5);
         if (p.pair_cnt) {
             // the CTA that delivers the last partial of a pair merges them all (no second kernel)
             __threadfence();
@@ -1199,12 +1259,14 @@ __device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& 
                 if (old == expected - 1) p.pair_cnt[pair] = 0;          // ready for the next call
             }
             soft_sync();
+            if (tid == 0) FDC_TSS(6);
             if (cx.flags[1])
                 merge_pair(p.ws_ml, p.ws_o, reinterpret_cast<__nv_bfloat16*>(p.out), pair, p.mmax, M, G, sg.s, sg.g, p.max_active, p.hq,
                            cx.flags[2], cx.flags[3]);
         }
     }
     soft_sync();                     // column state and Q^T are free again
+    if (tid == 0) { FDC_TS(9); FDC_TSS(8); }
     tc_fence_before();
     __syncwarp();
     if (!dead && lane == 0) mbar_arrive(cx.o_free);
@@ -1250,7 +1312,7 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, con
     cx.pre = cx.rflag + 4;
     cx.nact = cx.pre + p.batch + 1;
     cx.prev = cx.nact + p.batch;
-    cx.smask = reinterpret_cast<uint64_t*>(((uintptr_t)(cx.prev + p.batch + 1) + 7) & ~(uintptr_t)7);
+    cx.smask = reinterpret_cast<uint64_t*>(((uintptr_t)(cx.prev + p.batch + 1) + 15) & ~(uintptr_t)15);
     cx.sunion = cx.smask + 2 * MBUF;
     cx.mstaged = p.max_active * p.W <= MBUF;
     __shared__ int abort_flag, v_step_bits[4];
@@ -1258,6 +1320,7 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, con
     cx.v_steps = v_step_bits;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) FDC_TS(0);
     if (threadIdx.x == 0) {
         abort_flag = 0;
     }
@@ -1324,6 +1387,7 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, con
     tc_fence_after();
     const uint32_t tmem = split_only ? 0u : *reinterpret_cast<volatile uint32_t*>(tmem_holder);
     cx.tmem = tmem;
+    if (threadIdx.x == 0) FDC_TS(1);
     // Programmatic dependent launch: this grid may have been scheduled while the kernel before it in
     // the stream was still running, and the kernel after this one may be scheduled early in the same
     // way.  Ordinarily nothing of global memory is touched before the kernel ahead has completed, and
@@ -1335,6 +1399,7 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, con
     // Every thread passes the wait before the block ends, so grids complete in stream order.
     if (!p.early) asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    if (threadIdx.x == 0) FDC_TS(2);
     if (!p.early) issue_loads();
     bool active = true;                       // this CTA has units (uniform over the CTA)
     long long lo = 0, hi = 0;
@@ -1356,6 +1421,7 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, con
     __syncthreads();
     const long long total = scan_ntiles(cx.prev, p.batch, cx.pre);
     const long long U = total * p.hkv;
+    if (threadIdx.x == 0) FDC_TS(3);
     if (U == 0) active = false;
     cx.tpart = 0;
     cx.n_cta = p.n_cta;
@@ -1405,7 +1471,11 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, con
             }
         }
         __syncthreads();
+#ifdef FDC_EQUAL_SHARES
+        const bool one_part = false;                   // (development builds: always equal shares of the weighted length)
+#else
         const bool one_part = (long long)split_pairs * p.hkv <= p.n_cta;
+#endif
         if (one_part) {
             // every thread tries sizes of its own; the smallest that fits wins
             const uint32_t vmax = (uint32_t)vt_of(cx, split_max, split_max);
@@ -1481,6 +1551,7 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, con
         hi = cta_first_unit(blockIdx.x + 1, U, cx.n_cta);
     }
     if (lo >= hi || (int)blockIdx.x >= cx.n_cta) active = false;
+    if (threadIdx.x == 0) FDC_TS(4);
     if (split_only) {
         // this launch only computes the split and leaves it to the attention launches of the pass
         int32_t* mwr = p.split_memo;
@@ -1542,6 +1613,7 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, con
     // ---- teardown: everybody is done with TMEM before it is freed
     tc_fence_before();
     __syncthreads();
+    if (threadIdx.x == 0) FDC_TS(10);
     if (warp == W_QK && !split_only) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(TMEM_COLS) : "memory");
@@ -1549,6 +1621,16 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, con
 }
 
 }  // namespace
+
+#ifdef FDC_TRACE
+extern "C" int fdc_tr_read(long long* out)
+{
+    cudaDeviceSynchronize();
+    cudaMemcpyFromSymbol(out, g_tr, sizeof(long long) * 1024);
+    cudaMemcpyFromSymbol(out + 1024, g_ts, sizeof(long long) * 80);
+    return 0;
+}
+#endif
 
 namespace fdc {
 
