@@ -49,8 +49,9 @@ constexpr int W_PROD = NSOFT, W_QK = NSOFT + 1, W_AUX = NSOFT + 2, W_PV = NSOFT 
 constexpr int THREADS = (NSOFT + 4) * 32;
 constexpr uint32_t TMEM_COLS = 512;          // S^T buffers [0,256): 4 x 64 columns (2 x 128 for 128 query rows) | O^T [256,384) | sums [384,512)
 constexpr uint32_t TM_O = 256;
-constexpr uint32_t TM_L = 384;                // per-column sums of the softmax threads [384, 512)
+constexpr uint32_t TM_L = 384;                // column sums [384, 400): accumulator of the multiplication by ones (lane n: query column n)
 constexpr int PANEL = RROWS * 128;           // 128 rows x 128 bytes (64 bf16 columns)
+constexpr int ONES_BYTES = 2048;             // B operand of the column-sum multiplication: 16 x 16 bf16 ones (the footprint of its layout)
 constexpr int STAGE = (D / 64) * PANEL;      // one K (or V) stage: 128 rows x head_dim
 constexpr int MAXST = 4;                     // stages per ring at most
 constexpr float RAISE_LOG2 = 16.f;
@@ -85,7 +86,8 @@ constexpr int UW = 64;                       // words of a scene's union bitmap 
 constexpr int MIN_TILES = 8;                 // tiles per CTA below which fewer CTAs are used (small problems)
 constexpr int MIN_UNITS = MIN_TILES * W_PREFIX;   // the same as a weighted length
 static_assert(MIN_UNITS >= 2 * FDC_W_MASKED, "every part of a pair must contain the start of at least one tile");
-constexpr int MBUF = 512;                    // bitmap words of a scene kept in shared memory (max_active * W)
+constexpr int MBUF = 512;                    // bitmap words of a scene kept in shared memory (max_active * W): one buffer; 2 * MBUF for 128 query rows
+constexpr int MBUF_MAX = 1024;
 
 // ---------------------------------------------------------------- tcgen05 wrappers
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -188,12 +190,13 @@ struct Ctx {
     uint32_t k_full, k_empty, v_full, v_empty, s_full, s_free, p_full, pv_done, q_ready, o_free, app_done;
     int ns, s_stride;                // S^T buffers in TMEM (4 of 64 columns up to 64 query rows, else 2 of 128) and their distance
     uint32_t tmem;
-    unsigned char *kring, *vring, *qs, *ps;
+    unsigned char *kring, *vring, *qs, *ps, *ones;
     float *mneg, *alpha, *lred;      // [128] -reference per column, [128] rescale factors, [4][128] partial sums
     int *cmax, *flags;               // [128] column maxima (ordered ints), [4] flags of the raise path and the merge
     int* rflag;                      // [4] rflag[g & 3] == g: round g met a score far above its reference
     int *pre, *nact;                 // [batch + 1] tile prefix sums, [batch] active branches per scene
-    uint64_t* smask;                 // [2][MBUF] the current segment's scene bitmaps (when mstaged)
+    uint64_t* smask;                 // [2][mbuf] the current segment's scene bitmaps (when mstaged)
+    int mbuf;                        // words per buffer
     uint64_t* sunion;                // [2][UW] their OR over the scene's active branches (when mstaged and W <= UW)
     int mstaged;
     int n_cta;                       // CTAs that take part: at most the grid, at least MIN_UNITS tiles each
@@ -211,7 +214,7 @@ struct Ctx {
 // to shared memory at the start of a segment whenever they fit.
 __device__ __forceinline__ const uint64_t* mask_row(const AttnParams& p, const Ctx& cx, uint32_t seg, int s, int b)
 {
-    return cx.mstaged ? cx.smask + (seg & 1) * MBUF + (size_t)b * p.W : p.mask + ((size_t)s * p.max_active + b) * p.W;
+    return cx.mstaged ? cx.smask + (seg & 1) * cx.mbuf + (size_t)b * p.W : p.mask + ((size_t)s * p.max_active + b) * p.W;
 }
 // 16-byte asynchronous copy global -> shared (zero fill when !valid); completes with cp_async_wait_all.
 __device__ __forceinline__ void cp_async16(void* dst, const void* src, bool valid)
@@ -553,13 +556,18 @@ __device__ __noinline__ void append_rows(char* kc, char* vc, long long stride_sc
 __device__ __noinline__ uint64_t tile_seen_rows(const uint64_t* un, const uint64_t* mask0, int W, int P, int A, int tile)
 {
     if (un) return tile_rowmask(un, W, P, tile);
+    // (whole warp: the lanes share the branches and combine)
+    const int lane = threadIdx.x & 31;
     uint64_t um = 0ull;
-    for (int b = 0; b < A; ++b) um |= tile_rowmask(mask0 + (size_t)b * W, W, P, tile);
-    return um;
+    for (int b = lane; b < A; b += 32) um |= tile_rowmask(mask0 + (size_t)b * W, W, P, tile);
+    const uint32_t ul = __reduce_or_sync(0xffffffffu, (uint32_t)um);
+    const uint32_t uh = __reduce_or_sync(0xffffffffu, (uint32_t)(um >> 32));
+    return ((uint64_t)uh << 32) | ul;
 }
 
 // The auxiliary warp: with fdc_set_fused_append it writes the pass's new K/V rows that fall into
-// this CTA's tiles, then lets the producer go on to the tiles beyond the prefix.
+// this CTA's tiles, then lets the producer go on to the tiles beyond the prefix; after that one
+// of its threads issues the column-sum multiplications.
 __device__ __forceinline__ void aux_loop(const AttnParams& p, const Ctx& cx, long long lo, long long hi, int lane)
 {
     if (p.app_row) {
@@ -568,6 +576,51 @@ __device__ __forceinline__ void aux_loop(const AttnParams& p, const Ctx& cx, lon
                     reinterpret_cast<const char*>(p.app_v), p.tiles, p.ntile_max, p.max_active, p.hkv, p.rows, p.P, cx.pre, cx.nact, lo, hi,
                     p.status);
         if (lane == 0) mbar_arrive(cx.app_done);
+    }
+    // The column sums of P^T (the softmax denominators), taken by the tensor core beside every
+    // O^T += V^T P^T: P (128 query columns as rows, read from the same P^T buffer, which is laid out
+    // the same way for either operand) times 16 columns of ones, so that TMEM lane n of the accumulator
+    // holds sum_k P^T[k][n] of exactly the values that are multiplied with V.  For fewer than 128 query
+    // rows the multiplication reads on past the P^T buffer (shared memory of this CTA all the same):
+    // those rows of the result are never looked at, and a row depends on nothing but its own inputs.
+    // Issued from this warp so that the thread that issues the V multiplications is not slowed down;
+    // the same 16-row steps are left out, and both threads commit to the pv_done barrier.
+    const uint64_t ones_desc = smem_desc(smem_u32(cx.ones), PANEL, 1024);
+    const uint64_t p_desc0 = smem_desc(smem_u32(cx.ps), PANEL, 1024);
+    const uint32_t ones_lo = (uint32_t)ones_desc, ones_hi = (uint32_t)(ones_desc >> 32), p_lo0 = (uint32_t)p_desc0, p_hi = (uint32_t)(p_desc0 >> 32);
+    const uint32_t tm_l = cx.tmem + TM_L;
+    int s = 0;
+    uint32_t g = 0, seg = 0;
+    long long u = lo;
+    int ok = 1;
+    while (u < hi && ok) {
+        const Segment sg = decode_segment(u, hi, cx.pre, p.hkv, s);
+        if (lane == 0) {
+            const uint32_t idesc_sum = instr_desc(128, 16, 1);
+            const int ntile = sg.j1 - sg.j0;
+            bool good = true;
+            for (int t = 0; 2 * t < ntile && good; ++t, ++g) {
+                good = mbar_wait(cx.p_full + 8 * (g & 1), (g >> 1) & 1, cx.abortp, p.status);
+                if (good && t == 0 && seg > 0) good = mbar_wait(cx.o_free, (seg - 1) & 1, cx.abortp, p.status);
+                if (!good) break;
+                const uint32_t steps = (uint32_t)cx.v_steps[(g & 1) * 2] | ((uint32_t)cx.v_steps[(g & 1) * 2 + 1] << 4);
+                tc_fence_after();
+                const uint32_t pd = p_lo0 + (uint32_t)((((g & 1) & (cx.npb - 1)) * cx.p_buf) >> 4);
+                uint32_t acc = t > 0 ? 1u : 0u;
+#pragma unroll 1
+                for (int kk = 0; kk < 8; ++kk)
+                    if ((steps >> kk) & 1u) {
+                        umma2(tm_l, pd + kk * 128, p_hi, ones_lo, ones_hi, idesc_sum, acc);
+                        acc = 1u;
+                    }
+                umma_commit(cx.pv_done + 8 * (g & 1));
+            }
+            ok = good;
+        }
+        ok = __shfl_sync(0xffffffffu, ok, 0);
+        g = __shfl_sync(0xffffffffu, g, 0);
+        ++seg;
+        u = sg.next_u;
     }
 }
 
@@ -854,15 +907,7 @@ __device__ __noinline__ int raise_references(const RaiseArgs a)
         }
     }
     soft_sync();
-    if (flags[0]) {                                        // a reference moved: rescale sums and accumulator
-        for (int ch = 0; ch < a.nph / 8; ++ch) {
-            uint32_t lv[8];
-            tmem_ld<8>(a.l_addr + ch * 8, lv);
-            tmem_wait_ld();
-#pragma unroll
-            for (int i = 0; i < 8; ++i) lv[i] = __float_as_uint(__uint_as_float(lv[i]) * alpha[a.col0 + ch * 8 + i]);
-            tmem_st<8>(a.l_addr + ch * 8, lv);
-        }
+    if (flags[0]) {                                        // a reference moved: rescale the accumulators (column sums and O^T)
         if (a.rescale_o) {
             if (!dead && !mbar_wait(a.pv_bar, a.pv_parity, a.abortp, a.status)) dead = true;   // no MMA may be writing O^T
             dead = __any_sync(0xffffffffu, dead);
@@ -875,6 +920,15 @@ __device__ __noinline__ int raise_references(const RaiseArgs a)
 #pragma unroll
                     for (int i = 0; i < 8; ++i) ov[i] = __float_as_uint(__uint_as_float(ov[i]) * alpha[a.col0 + ch * 8 + i]);
                     tmem_st<8>(a.o_addr + ch * 8, ov);
+                }
+                if (a.col0 == 0) {                          // the column sums: TMEM lane n belongs to query column n
+                    uint32_t lv[8];
+                    tmem_ld<8>(a.l_addr, lv);
+                    tmem_wait_ld();
+                    const float al = alpha[threadIdx.x & 127];
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) lv[i] = __float_as_uint(__uint_as_float(lv[i]) * al);
+                    tmem_st<8>(a.l_addr, lv);
                 }
             }
         }
@@ -932,10 +986,10 @@ __device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& 
                     qv[i] = qg[((((size_t)sg.s * p.max_active + b) * p.hq + (size_t)sg.g * G + hg) * D) / 8 + ch];
                 }
             }
-            uint64_t mv[MBUF / (NSOFT * 32)];
+            uint64_t mv[MBUF_MAX / (NSOFT * 32)];
             const int nw = cx.mstaged ? p.max_active * p.W : 0;
 #pragma unroll
-            for (int i = 0; i < MBUF / (NSOFT * 32); ++i) {
+            for (int i = 0; i < MBUF_MAX / (NSOFT * 32); ++i) {
                 const int idx = tid + i * (NSOFT * 32);
                 mv[i] = idx < nw ? p.mask[(size_t)sg.s * p.max_active * p.W + idx] : 0ull;
             }
@@ -946,29 +1000,22 @@ __device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& 
                 if (n < np) *reinterpret_cast<uint4*>(cx.qs + (ch >> 3) * cx.q_panel + n * 128 + (((ch & 7) ^ (n & 7)) << 4)) = qv[i];
             }
 #pragma unroll
-            for (int i = 0; i < MBUF / (NSOFT * 32); ++i) {
+            for (int i = 0; i < MBUF_MAX / (NSOFT * 32); ++i) {
                 const int idx = tid + i * (NSOFT * 32);
-                if (idx < nw) cx.smask[(seg & 1) * MBUF + idx] = mv[i];
+                if (idx < nw) cx.smask[(seg & 1) * cx.mbuf + idx] = mv[i];
             }
         }
         if (cx.mstaged && p.W <= UW && !published) {
             // OR of the scene's bitmaps: the rows that some branch may see (the others are cleared in V)
             soft_sync();                              // everybody's share of the bitmaps is in place
             if (tid < p.W) {
-                const uint64_t* mb = cx.smask + (seg & 1) * MBUF + tid;
+                const uint64_t* mb = cx.smask + (seg & 1) * cx.mbuf + tid;
                 uint64_t un = 0ull;
                 for (int b = 0; b < A; ++b) un |= mb[(size_t)b * p.W];
                 cx.sunion[(seg & 1) * UW + tid] = un;
             }
         }
         if (tid < np) cx.mneg[tid] = UNSET;
-        {
-            uint32_t z[8];
-#pragma unroll
-            for (int i = 0; i < 8; ++i) z[i] = 0u;
-            for (int ch = 0; ch < nch; ++ch) tmem_st<8>(l_addr + ch * 8, z);      // column sums start at 0
-            tmem_wait_st();
-        }
         if (!published) {
             fence_async_smem();
             __syncwarp();
@@ -1003,7 +1050,7 @@ __device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& 
                 // The next segment's queries (and its scene's bitmaps, into the other buffer) are copied
                 // asynchronously; the latency hides behind this round, the drain and the partial write.
                 prefetch_next_segment(reinterpret_cast<const uint4*>(p.q), p.mask, p.max_active, p.W, p.hq, G, p.hkv, cx.pre, cx.nact, cx.qs,
-                                      cx.q_panel, cx.mstaged ? cx.smask + ((seg + 1) & 1) * MBUF : nullptr, sg.next_u, hi, sg.s);
+                                      cx.q_panel, cx.mstaged ? cx.smask + ((seg + 1) & 1) * cx.mbuf : nullptr, sg.next_u, hi, sg.s);
                 prefetched = 1;
             }
             // The P^T buffer is still being read until the PV that used it last (two rounds ago, or the
@@ -1058,9 +1105,8 @@ __device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& 
                 float emax = 0.f;
 #pragma unroll 1
                 for (int ch = 0; ch < nch; ++ch) {
-                    uint32_t sv[8], lv[8];
+                    uint32_t sv[8];
                     tmem_ld<8>(s_addr + ch * 8, sv);
-                    tmem_ld<8>(l_addr + ch * 8, lv);
                     const float4 m0 = *reinterpret_cast<const float4*>(cx.mneg + col0 + ch * 8);
                     const float4 m1 = *reinterpret_cast<const float4*>(cx.mneg + col0 + ch * 8 + 4);
                     const float mn[8] = {m0.x, m0.y, m0.z, m0.w, m1.x, m1.y, m1.z, m1.w};
@@ -1077,22 +1123,17 @@ __device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& 
                         e[i] = fast_exp2(fmaf(__uint_as_float(sv[i]), c, mn[i]));
                         emax = fmaxf(emax, e[i]);
                     }
-                    // P^T goes to the tensor core as bf16; the column sums add up the SAME rounded values, so
-                    // numerator and denominator of the softmax stay consistent (the rounding cancels where a
-                    // few terms dominate)
+                    // P^T goes to the tensor core as bf16.  The column sums (the softmax denominators) are taken by
+                    // the tensor core too, from the SAME rounded values (a multiplication of P^T by ones beside
+                    // every O^T += V^T P^T), so numerator and denominator stay consistent: the rounding cancels
+                    // where a few terms dominate.
                     uint32_t pk[4];
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        pk[j] = pack2(e[2 * j], e[2 * j + 1]);
-                        lv[2 * j] = __float_as_uint(__uint_as_float(lv[2 * j]) + __uint_as_float(pk[j] << 16));
-                        lv[2 * j + 1] = __float_as_uint(__uint_as_float(lv[2 * j + 1]) + __uint_as_float(pk[j] & 0xffff0000u));
-                    }
-                    tmem_st<8>(l_addr + ch * 8, lv);
+                    for (int j = 0; j < 4; ++j) pk[j] = pack2(e[2 * j], e[2 * j + 1]);
                     const int cidx = (col0 >> 3) + ch;                 // 16-byte chunk of the P^T row
                     *reinterpret_cast<uint4*>(prow + (cidx >> 3) * PANEL + (((cidx & 7) ^ (krow & 7)) << 4)) =
                         make_uint4(pk[0], pk[1], pk[2], pk[3]);
                 }
-                tmem_wait_st();
                 if (emax > 65536.f) {                                  // 2^16 above the reference: note it for round g + 2
                     cx.rflag[g & 3] = (int)g;
                     if (!(emax < 1.0e30f)) atomicOr(p.status, FDC_DEV_SCORE_RANGE);     // beyond 2^100 (or inf / nan)
@@ -1153,7 +1194,7 @@ __device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& 
             int s2 = sg.s;
             const Segment nx = decode_segment(sg.next_u, hi, cx.pre, p.hkv, s2);
             if (tid < p.W) {
-                const uint64_t* mb = cx.smask + ((seg + 1) & 1) * MBUF + tid;
+                const uint64_t* mb = cx.smask + ((seg + 1) & 1) * cx.mbuf + tid;
                 uint64_t un = 0ull;
                 const int A2 = cx.nact[nx.s];
                 for (int b = 0; b < A2; ++b) un |= mb[(size_t)b * p.W];
@@ -1170,29 +1211,14 @@ __device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& 
     wait_u(cx.pv_done + 8 * (last & 1), (last >> 1) & 1);
     tc_fence_after();
     if (tid == 0) { FDC_TS(8); FDC_TSS(3); }
-    // column sums over the warp's 32 rows by transpose-reduce: lane i < 8 ends up with column i's sum
-#pragma unroll 1
-    for (int ch = 0; ch < nch; ++ch) {
+    // column sums: TMEM lane n of the accumulator of the multiplication by ones
+    if (part == 0) {
         uint32_t lv[8];
-        tmem_ld<8>(l_addr + ch * 8, lv);
+        tmem_ld<8>(cx.tmem + lane_base + TM_L, lv);
         tmem_wait_ld();
-        float v[8];
-#pragma unroll
-        for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(lv[i]);
-#pragma unroll
-        for (int o = 16; o >= 8; o >>= 1)
-#pragma unroll
-            for (int i = 0; i < 8; ++i) v[i] += __shfl_xor_sync(0xffffffffu, v[i], o);
-#pragma unroll
-        for (int k = 4; k >= 1; k >>= 1) {
-            const bool up = (lane & k) != 0;
-#pragma unroll
-            for (int i = 0; i < k; ++i) {
-                const float recv = __shfl_xor_sync(0xffffffffu, up ? v[i] : v[i + k], k);
-                v[i] = (up ? v[i + k] : v[i]) + recv;
-            }
-        }
-        if (lane < 8) cx.lred[q4 * 128 + col0 + ch * 8 + lane] = v[0];
+        cx.lred[krow] = __uint_as_float(lv[0]);
+    } else {
+        cx.lred[part * 128 + krow] = 0.f;
     }
     soft_sync();
     const int pair = sg.s * p.hkv + sg.g;
@@ -1288,7 +1314,8 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, con
     cx.vring = cx.kring + (size_t)nk * STAGE;
     cx.ps = cx.vring + (size_t)nv * STAGE;
     cx.qs = cx.ps + npb * cx.p_buf;
-    uint64_t* bars = reinterpret_cast<uint64_t*>(cx.qs + (D / 64) * cx.q_panel);
+    cx.ones = cx.qs + (D / 64) * cx.q_panel;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(cx.ones + ONES_BYTES);
     cx.k_full = smem_u32(bars);
     cx.k_empty = cx.k_full + 8 * MAXST;
     cx.v_full = cx.k_empty + 8 * MAXST;
@@ -1313,8 +1340,9 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, con
     cx.nact = cx.pre + p.batch + 1;
     cx.prev = cx.nact + p.batch;
     cx.smask = reinterpret_cast<uint64_t*>(((uintptr_t)(cx.prev + p.batch + 1) + 15) & ~(uintptr_t)15);
-    cx.sunion = cx.smask + 2 * MBUF;
-    cx.mstaged = p.max_active * p.W <= MBUF;
+    cx.mbuf = np_max > 64 ? MBUF_MAX : MBUF;
+    cx.sunion = cx.smask + 2 * cx.mbuf;
+    cx.mstaged = p.max_active * p.W <= cx.mbuf;
     __shared__ int abort_flag, v_step_bits[4];
     cx.abortp = &abort_flag;
     cx.v_steps = v_step_bits;
@@ -1325,6 +1353,10 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, con
         abort_flag = 0;
     }
     if (threadIdx.x < 4) cx.rflag[threadIdx.x] = -1;
+    if (threadIdx.x < ONES_BYTES / 4 && !split_only) {
+        reinterpret_cast<uint32_t*>(cx.ones)[threadIdx.x] = 0x3F803F80u;          // bf16 1.0 twice
+        fence_async_smem();
+    }
     // The layers of one forward pass see the same per-scene counts, so the work split is made once
     // per pass (a launch of this kernel with split_only set) and kept in the memo, with the counts it
     // was computed from.  The memo's loads and those of the counts are all issued before the first
@@ -1369,7 +1401,7 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, con
         }
         for (int i = 0; i < 2; ++i) {
             mbar_init(cx.p_full + 8 * i, NSOFT);
-            mbar_init(cx.pv_done + 8 * i, 1);
+            mbar_init(cx.pv_done + 8 * i, 2);              // the V multiplications and the column sums
         }
         mbar_init(cx.q_ready, NSOFT);
         mbar_init(cx.o_free, NSOFT);
@@ -1643,8 +1675,8 @@ static int launch_tc(const AttnParams& p, int head_dim, cudaStream_t st, int spl
     const int np_max = p.mmax <= 32 ? 32 : (p.mmax <= 64 ? 64 : 128);
     const int p_buf = ((np_max + 63) / 64) * PANEL;
     const int npb = np_max > 64 ? 1 : 2;          // 128 query rows: one P^T buffer, so that four stages still fit
-    const size_t fixed = 1024 + (size_t)npb * p_buf + (size_t)(D / 64) * np_max * 128 + 8 * (5 * MAXST + 16) + 16 +
-                         4 * (128 + 128 + 512 + 128 + 8) + sizeof(int) * (3 * p.batch + 2) + 8 * (2 * MBUF + 2 * UW + 2) + 64;
+    const size_t fixed = 1024 + (size_t)npb * p_buf + (size_t)(D / 64) * np_max * 128 + ONES_BYTES + 8 * (5 * MAXST + 16) + 16 +
+                         4 * (128 + 128 + 512 + 128 + 8) + sizeof(int) * (3 * p.batch + 2) + 8 * (2 * (np_max > 64 ? MBUF_MAX : MBUF) + 2 * UW + 2) + 64;
     int stages = (int)((227 * 1024 - 256 - fixed) / STAGE);
     if (stages > 2 * MAXST) stages = 2 * MAXST;
     if (stages < 4) return FDC_ERR_SHAPE;

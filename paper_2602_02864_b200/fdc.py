@@ -110,6 +110,8 @@ def _ptr(t) -> Optional[int]:
 
 
 def _stream(stream) -> Optional[int]:
+    """cudaStream_t of a torch stream / raw handle; None = torch's current stream (looked up per call:
+    callers with a hot loop pass the handle, see DecodeSession.use_stream)."""
     if stream is None:
         return torch.cuda.current_stream().cuda_stream
     return int(stream.cuda_stream) if hasattr(stream, "cuda_stream") else int(stream)
@@ -286,6 +288,7 @@ class DecodeSession:
         self.ws_bytes = 0
         self.kv = None
         self._append_refs = None
+        self.stream = None                   # None: torch's current stream at every call
 
     def close(self):
         if self.plan:
@@ -298,6 +301,14 @@ class DecodeSession:
         except Exception:
             pass
 
+    def use_stream(self, stream) -> None:
+        """Fixes the stream of all later calls (a torch stream, a raw cudaStream_t or None for "torch's
+        current stream at every call"): the per-call look-up costs more than a small launch."""
+        self.stream = None if stream is None else _stream(stream)
+
+    def _st(self, stream):
+        return self.stream if stream is None else stream
+
     def bind_cache(self, k: torch.Tensor, v: torch.Tensor, hq: int) -> None:
         self.kv = kv_desc_from_tensors(k, v, hq)
         self._k, self._v = k, v
@@ -309,22 +320,22 @@ class DecodeSession:
     def init(self, lens: Optional[torch.Tensor], stream=None) -> None:
         """lens: int32 device tensor [batch][n_nodes] or None (fields run to their slot)."""
         self._lens = lens
-        fdc_state_init(self.plan, self.batch, lens, self.state, stream)
+        fdc_state_init(self.plan, self.batch, lens, self.state, self._st(stream))
 
     def frontier(self, finish: Optional[torch.Tensor] = None, stream=None) -> None:
         fdc_frontier(self.plan, self.batch, self.state, finish, self.n_active, self.node, self.tok_idx, self.kv_row,
-                     self.pos_id, self.all_done, stream)
+                     self.pos_id, self.all_done, self._st(stream))
 
     def build_masks(self, stream=None) -> None:
-        fdc_build_masks(self.plan, self.batch, self.state, self.mask, self.umask, self.tiles, self.ntiles, stream)
+        fdc_build_masks(self.plan, self.batch, self.state, self.mask, self.umask, self.tiles, self.ntiles, self._st(stream))
 
     def kv_append(self, layer, k_new, v_new, stream=None) -> None:
-        fdc_kv_append(self.plan, self.kv, layer, self.n_active, self.kv_row, k_new, v_new, stream)
+        fdc_kv_append(self.plan, self.kv, layer, self.n_active, self.kv_row, k_new, v_new, self._st(stream))
         self._append_refs = (k_new, v_new)      # a recorded (fused) append reads them in the next decode_attn
 
     def decode_attn(self, layer, q, out, scale, stream=None) -> None:
         fdc_decode_attn(self.plan, self.kv, layer, self.n_active, self.mask, self.tiles, self.ntiles, q, out, scale,
-                        self.workspace, self.ws_bytes, stream)
+                        self.workspace, self.ws_bytes, self._st(stream))
         self._append_refs = None
 
     def set_fused_append(self, on: bool) -> None:
