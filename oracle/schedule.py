@@ -3,7 +3,7 @@
 TEST INFRASTRUCTURE ONLY (see the package docstring).  Notation follows the paper:
 G = (V, E), d_v = remaining unfinished prerequisites of v, S = ready set.
 
-Readings taken where the paper is silent (all listed in the design notes):
+Readings taken where the paper is silent (Sec. 3.2 - 3.3 leave these open):
   * a newly ready field first decodes in the NEXT forward pass (Alg. 1: decoding is the
     first statement of the next loop iteration);
   * within a pass fields are packed in ascending node id;

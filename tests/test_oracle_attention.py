@@ -183,3 +183,25 @@ def test_threads_do_not_change_result():
     vis = rng.random((4, 100)) < 0.7
     vis[:, 0] = True
     assert (oatt.attention(q, K, V, vis, 0.25, nthreads=1) == oatt.attention(q, K, V, vis, 0.25, nthreads=4)).all()
+
+
+def test_oracle_run_places_fixed_rows_by_hand_example():
+    """OracleRun.write_fixed: the pre-filled field-name rows (Sec. 3.3, Fig. 3: "pre-filled") go to the
+    head of their fields' slots.  Hand example: slots of 3, 4 and 3 rows after a prefix of 2 rows, so
+    field 0 starts at row 2, field 1 at row 5, field 2 at row 9; one fixed row in field 0 (row 2), none
+    in field 1, two in field 2 (rows 9 and 10).  The i-th fixed row carries the value i + 1."""
+    from oracle import run as orun
+    lens = np.array([[2, 3, 3]], np.int32)
+    o = orun.OracleRun(3, [], [3, 4, 3], [1, 0, 2], 2, lens, layers=2, hq=2, hkv=2, head_dim=4, scale=0.5, max_active=3)
+    K = np.zeros((1, 2, 3, 4), np.float32)
+    for i in range(3):
+        K[:, :, i] = i + 1
+    o.write_fixed(1, K, -K)
+    want = {2: 1.0, 9: 2.0, 10: 3.0}
+    for r in range(o.R):
+        for h in range(2):
+            if r in want:
+                assert (o.K[0, 1, h, r] == want[r]).all() and (o.V[0, 1, h, r] == -want[r]).all()
+            else:
+                assert np.isnan(o.K[0, 1, h, r]).all() and np.isnan(o.V[0, 1, h, r]).all()
+    assert np.isnan(o.K[0, 0]).all()                     # the other layer untouched

@@ -190,6 +190,30 @@ def test_eq1_hand_example():
     assert n_checked == 7
 
 
+def test_tile_list_and_union_bitmap_hand_example():
+    """pass_tables' tile list, union bitmap and branch bitmaps against a hand-worked case: a prefix
+    that is no tile multiple, a tile that holds nothing but padding, a partial last tile."""
+    n, edges, cap, lens, P = 3, [(0, 2)], [140, 70, 30], [5, 8, 2], 70
+    passes = sch.simulate(n, edges, lens)
+    assert len(passes) == 8 and passes[5] == [(1, 5), (2, 0)] and passes[7] == [(1, 7)]
+    n_checked = 0
+    for line in open(os.path.join(GOLD, "tile_list_example.txt")):
+        if not line.strip() or line.startswith("#"):
+            continue
+        left, right = line.split(":")
+        f = left.split()
+        want = [int(x) for x in right.split()]
+        tab = sch.pass_tables(n, edges, cap, lens, [0] * n, P, passes[int(f[1])])
+        if f[2] == "tiles":
+            assert tab["tiles"].tolist() == want, line
+        elif f[2] == "umask":
+            assert [int(x) for x in tab["umask"]] == want, line
+        else:
+            assert [int(x) for x in tab["mask"][int(f[3])]] == want, line
+        n_checked += 1
+    assert n_checked == 7
+
+
 def test_mask_invariants_random():
     for seed in range(60):
         w = wl.random_template(9000 + seed, n_nodes=2 + seed % 8, fixed_hi=seed % 3, prefix_len=seed % 130,
@@ -237,7 +261,7 @@ def test_chain_mask_is_lower_triangular():
 
 
 def test_workload_shapes():
-    """The synthetic configurations have the sizes the benchmark's configs state."""
+    """The synthetic configurations have the stated sizes (Sec. 3.1: a CoT of 300-500 tokens, fixed slots)."""
     w1 = wl.cfg1_7b()
     assert (w1.layers, w1.hq, w1.hkv, w1.head_dim, w1.batch, w1.prefix_len) == (28, 28, 4, 128, 1, 2048)
     assert w1.lens.min() >= 32 and w1.lens.max() <= 64 and w1.cot_rows == 512

@@ -6,8 +6,10 @@ fail once the KV pool owns the GPU), or a plugin-style host whose per-step call 
 allocate.  For them the library carries its own 16 MiB scratch buffer and this entry point
 takes no workspace argument.  The test drives it through the C ABI and checks that it gives
 what fdc_decode_attn gives with a caller-owned workspace, on two calls in a row (the buffer is
-shared and keeps the previous call's contents, so the second call sees stale data), and that
-a problem too large for the built-in buffer is refused before anything is launched.
+shared and keeps the previous call's contents, so the second call sees stale data), that its
+result also matches the float64 CPU checker, that the amount of free device memory is the same
+before and after a series of such calls (the property the entry point exists for), and that a
+problem too large for the built-in buffer is refused before anything is launched.
 
 Collected last on purpose (file name): a run that stops at the first failure has then already
 run every other test.  It does not depend on the other tests having run or not.
@@ -81,6 +83,51 @@ def test_static_scratch_matches_caller_workspace_twice_in_a_row(make):
                 rel = np.sqrt((err ** 2).sum(-1)) / np.sqrt((b[s, :A].astype(np.float64) ** 2).sum(-1))
                 assert err.max() <= BF16_MAX_ABS and rel.max() <= BF16_REL_L2
     assert fdc.fdc_launch_count() > launches0
+    assert sess.status() == 0
+    sess.close()
+
+
+def test_static_calls_take_no_device_memory_and_match_the_checker():
+    """After a first call (which may load the library's device image and looks up the buffer's
+    address) further calls must leave cudaMemGetInfo's free figure exactly where it was; and what
+    they compute is the checker's masked attention, within the bf16 tolerance."""
+    from paper_2602_02864_b200 import fdc
+    from harness import check_close, make_oracle
+    w = wl.cfg2_batched(layers=1, batch=2)
+    device = "cuda"
+    oracle = make_oracle(w)
+    sess = fdc.DecodeSession(w.n_nodes, w.edges, w.slot_cap, w.n_fixed, w.prefix_len, w.max_active, w.batch, device)
+    k, v = alloc_cache(w, device)
+    write_prefix(w, k, v, oracle)
+    sess.bind_cache(k, v, w.hq)
+    sess.init(torch.from_numpy(w.lens).to(device))
+    outs = [torch.full((w.batch, w.max_active, w.hq, w.head_dim), 7.0, dtype=w.torch_dtype, device=device) for _ in range(3)]
+    steps = []
+    for step in range(3):                       # everything torch allocates is allocated before the measurement
+        steps.append(wl.step_qkv(w, step, 0, device))
+
+    def one_pass(step):
+        q, kn, vn = steps[step]
+        sess.frontier(None)
+        sess.build_masks()
+        sess.kv_append(0, kn, vn)
+        fdc.fdc_decode_attn_static(sess.plan, sess.kv, 0, sess.n_active, sess.mask, sess.tiles, sess.ntiles, q, outs[step],
+                                   w.softmax_scale)
+
+    one_pass(0)                                 # start-up call
+    torch.cuda.synchronize()
+    free0 = torch.cuda.mem_get_info()[0]
+    one_pass(1)
+    one_pass(2)
+    torch.cuda.synchronize()
+    assert torch.cuda.mem_get_info()[0] == free0
+    for step in range(3):
+        q, kn, vn = steps[step]
+        oracle.append(step, 0, f32(kn), f32(vn))
+        ref = oracle.attend(step, 0, f32(q))
+        for s in range(w.batch):
+            A = len(oracle.active(s, step))
+            check_close(f32(outs[step])[s, :A], ref[s, :A], w.dtype, f"static call, pass {step} scene {s}")
     assert sess.status() == 0
     sess.close()
 
