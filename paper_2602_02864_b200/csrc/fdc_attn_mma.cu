@@ -421,10 +421,10 @@ PFN_cuTensorMapEncodeTiled get_encode()
 struct MapKey {
     const void* base;
     int64_t ss, sh, sr;
-    int32_t batch, hkv, rows, d, box_rows;
+    int32_t batch, hkv, rows, d, box_rows, dev;
     bool operator==(const MapKey& o) const
     {
-        return base == o.base && ss == o.ss && sh == o.sh && sr == o.sr && batch == o.batch && hkv == o.hkv && rows == o.rows && d == o.d && box_rows == o.box_rows;
+        return dev == o.dev && base == o.base && ss == o.ss && sh == o.sh && sr == o.sr && batch == o.batch && hkv == o.hkv && rows == o.rows && d == o.d && box_rows == o.box_rows;
     }
 };
 struct MapCache {
@@ -435,7 +435,9 @@ MapCache g_maps;
 
 int get_map(const void* base, const AttnParams& p, int d, int box_rows, CUtensorMap* out)
 {
-    MapKey key{base, p.stride_scene, p.stride_head, p.stride_row, p.batch, p.hkv, p.rows, d, box_rows};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return FDC_ERR_CUDA;
+    MapKey key{base, p.stride_scene, p.stride_head, p.stride_row, p.batch, p.hkv, p.rows, d, box_rows, dev};
     std::lock_guard<std::mutex> lk(g_maps.mu);
     for (auto& it : g_maps.items)
         if (it.first == key) {
@@ -471,14 +473,11 @@ int launch_t(const AttnParams& p, cudaStream_t st)
     if (nstage > 16) nstage = 16;
     if (nstage < 2) return FDC_ERR_SHAPE;
     const size_t smem = fixed + (size_t)nstage * STAGE_BYTES;
-    static size_t attr_smem = 0;
-    if (smem > attr_smem) {
-        cudaError_t e = cudaFuncSetAttribute(attn_mma_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return set_cuda_error(e);
-        attr_smem = smem;
-    }
+    static size_t attr_smem[kMaxDevices] = {};
+    int rc = raise_dynamic_smem(reinterpret_cast<const void*>(attn_mma_kernel<D>), smem, attr_smem);
+    if (rc) return rc;
     alignas(64) CUtensorMap tk, tv;
-    int rc = get_map(p.k, p, D, SROWS, &tk);
+    rc = get_map(p.k, p, D, SROWS, &tk);
     if (rc) return rc;
     rc = get_map(p.v, p, D, SROWS, &tv);
     if (rc) return rc;

@@ -4,7 +4,7 @@
 // row may see.  Used for the fp32 configuration and as the fallback for every other one.
 #include <cuda_bf16.h>
 
-#include "fdc_internal.h"
+#include "fdc_attn_common.cuh"
 
 using namespace fdc;
 
@@ -32,29 +32,6 @@ __device__ __forceinline__ float warp_sum(float x)
 #pragma unroll
     for (int o = 16; o; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
     return x;
-}
-
-// Exclusive prefix sums of ntiles over scenes into smem pre[0..batch]; returns total.
-__device__ int scan_ntiles(const int32_t* __restrict__ ntiles, int batch, int* pre)
-{
-    if (threadIdx.x < 32) {
-        int carry = 0;
-        for (int b0 = 0; b0 < batch; b0 += 32) {
-            int i = b0 + threadIdx.x;
-            int x = i < batch ? ntiles[i] : 0;
-            int inc = x;
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                int y = __shfl_up_sync(0xffffffffu, inc, o);
-                if ((int)threadIdx.x >= o) inc += y;
-            }
-            if (i < batch) pre[i] = carry + inc - x;
-            carry += __shfl_sync(0xffffffffu, inc, 31);
-        }
-        if (threadIdx.x == 0) pre[batch] = carry;
-    }
-    __syncthreads();
-    return pre[batch];
 }
 
 template <typename T, int D>
@@ -264,12 +241,9 @@ int launch_ref_t(const AttnParams& p, cudaStream_t st)
     size_t smem = sizeof(float) * ((size_t)64 * (D + 1) + 64 * D + 2 * (size_t)p.mmax * D + kWarps * 64 + 2 * p.mmax) +
                   sizeof(int) * (p.batch + 1);
     if (smem > 227 * 1024) return FDC_ERR_SHAPE;
-    static size_t attr_smem = 0;
-    if (smem > attr_smem) {
-        cudaError_t e = cudaFuncSetAttribute(attn_ref_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return set_cuda_error(e);
-        attr_smem = smem;
-    }
+    static size_t attr_smem[kMaxDevices] = {};
+    const int rcs = raise_dynamic_smem(reinterpret_cast<const void*>(attn_ref_kernel<T, D>), smem, attr_smem);
+    if (rcs) return rcs;
     attn_ref_kernel<T, D><<<p.n_cta, kThreads, smem, st>>>(p);
     note_launch();
     cudaError_t e = cudaGetLastError();

@@ -170,7 +170,35 @@ __device__ __forceinline__ void tmem_st(uint32_t taddr, const uint32_t (&v)[N])
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
+// Barrier of the softmax warps (a named barrier).  Every call site is reached by all sixteen warps
+// the same number of times whatever happens: a warp whose bounded wait ran out goes on without
+// waiting but still takes every one of these.
 __device__ __forceinline__ void soft_sync() { asm volatile("bar.sync 1, %0;" ::"n"(NSOFT * 32) : "memory"); }
+
+// The barrier inside the reference-raising path.  Whether a warp enters that path in a given round
+// depends on data (a note left two rounds earlier), which a warp that no longer waits for anything
+// may read too early; a named barrier there could then be waited at for ever.  So this one is an
+// mbarrier with a bounded wait, one arrival per warp: the worst a straying warp can cause is that the
+// others give up too (FDC_DEV_TIMEOUT).
+static __device__ __noinline__ void raise_sync_slow(uint32_t bar, uint64_t tok, volatile int* abort_flag, int32_t* status)
+{
+    for (uint32_t i = 0; i < (1u << 18); ++i) {
+        uint32_t ok;
+        asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(ok) : "r"(bar), "l"(tok) : "memory");
+        if (ok) return;
+        if ((i & 255u) == 255u && *abort_flag) return;
+    }
+    *abort_flag = 1;
+    atomicOr(status, FDC_DEV_TIMEOUT);
+}
+__device__ __forceinline__ void raise_sync(uint32_t bar, volatile int* abort_flag, int32_t* status)
+{
+    __syncwarp();
+    uint64_t tok = 0;
+    if ((threadIdx.x & 31) == 0) asm volatile("mbarrier.arrive.shared::cta.b64 %0, [%1];" : "=l"(tok) : "r"(bar) : "memory");
+    tok = __shfl_sync(0xffffffffu, tok, 0);
+    raise_sync_slow(bar, tok, abort_flag, status);
+}
 
 __device__ __forceinline__ uint32_t pack2(float lo, float hi)
 {
@@ -185,9 +213,31 @@ __device__ __forceinline__ int ord_of(float x)
 }
 __device__ __forceinline__ float ord_to(int i) { return __int_as_float(i ^ ((i >> 31) & 0x7fffffff)); }
 
+// Small per-CTA state in static shared memory.  The raise path finds its barrier from the address of
+// the abort flag (it is handed that address anyway).
+struct __align__(8) CtaFlags {
+    uint64_t raise_bar;              // mbarrier of the reference-raising path (raise_sync)
+    int abort_flag;                  // a bounded wait ran out somewhere in the CTA
+    int v_steps[4];
+};
+constexpr uint32_t RAISE_BAR_BEFORE_ABORT_FLAG = 8;
+static_assert(offsetof(CtaFlags, abort_flag) - offsetof(CtaFlags, raise_bar) == RAISE_BAR_BEFORE_ABORT_FLAG, "layout");
+
 // Everything a role needs to find its barriers and buffers.
 struct Ctx {
-    uint32_t k_full, k_empty, v_full, v_empty, s_full, s_free, p_full, pv_done, q_ready, o_free, app_done;
+    // mbarriers: one base address, fixed offsets (kept as functions so that a single register serves them all)
+    uint32_t bar0;
+    __device__ __forceinline__ uint32_t k_full() const { return bar0; }
+    __device__ __forceinline__ uint32_t k_empty() const { return bar0 + 8 * MAXST; }
+    __device__ __forceinline__ uint32_t v_full() const { return bar0 + 16 * MAXST; }
+    __device__ __forceinline__ uint32_t v_empty() const { return bar0 + 24 * MAXST; }
+    __device__ __forceinline__ uint32_t s_full() const { return bar0 + 32 * MAXST; }
+    __device__ __forceinline__ uint32_t s_free() const { return bar0 + 32 * MAXST + 32; }
+    __device__ __forceinline__ uint32_t p_full() const { return bar0 + 32 * MAXST + 64; }
+    __device__ __forceinline__ uint32_t pv_done() const { return bar0 + 32 * MAXST + 80; }
+    __device__ __forceinline__ uint32_t q_ready() const { return bar0 + 32 * MAXST + 96; }
+    __device__ __forceinline__ uint32_t o_free() const { return bar0 + 32 * MAXST + 104; }
+    __device__ __forceinline__ uint32_t app_done() const { return bar0 + 32 * MAXST + 112; }
     int ns, s_stride;                // S^T buffers in TMEM (4 of 64 columns up to 64 query rows, else 2 of 128) and their distance
     uint32_t tmem;
     unsigned char *kring, *vring, *qs, *ps, *ones;
@@ -370,7 +420,7 @@ __device__ __forceinline__ void producer_loop(const AttnParams& p, const Ctx& cx
     int q_hold = p.early;                            // after the wait, the first pair's queries go ahead of further K/V requests
     while ((ck.live || cv.live) && ok) {
         if (!app_ok && waited) {
-            const int done = lane == 0 ? (int)mbar_try(cx.app_done, 0) : 0;
+            const int done = lane == 0 ? (int)mbar_try(cx.app_done(), 0) : 0;
             app_ok = __shfl_sync(0xffffffffu, done, 0);
         }
         // Rows beyond the prefix may have been written by the kernel ahead (fdc_kv_append) or are written
@@ -378,7 +428,7 @@ __device__ __forceinline__ void producer_loop(const AttnParams& p, const Ctx& cx
         if (q_hold && waited) {
             // The queries are requested right after the wait; whatever this SM requests before them
             // arrives before them.  The stages requested ahead of the wait keep the first rounds fed.
-            const int done = lane == 0 ? (int)mbar_try(cx.q_ready, 0) : 0;
+            const int done = lane == 0 ? (int)mbar_try(cx.q_ready(), 0) : 0;
             q_hold = !__shfl_sync(0xffffffffu, done, 0);
         }
         const bool hold_all = q_hold && waited;
@@ -386,19 +436,19 @@ __device__ __forceinline__ void producer_loop(const AttnParams& p, const Ctx& cx
         const bool hold_v = hold_all || (!(app_ok && waited) && cv.live && cursor_beyond_prefix(cv, p.P));
         int rk = 0, rv = 0;
         if (lane == 0) {
-            rk = ck.live && !hold_k && mbar_try(cx.k_empty + 8 * ck.st, ck.ph ^ 1);
-            rv = cv.live && !hold_v && mbar_try(cx.v_empty + 8 * cv.st, cv.ph ^ 1);
+            rk = ck.live && !hold_k && mbar_try(cx.k_empty() + 8 * ck.st, ck.ph ^ 1);
+            rv = cv.live && !hold_v && mbar_try(cx.v_empty() + 8 * cv.st, cv.ph ^ 1);
         }
         rk = __shfl_sync(0xffffffffu, rk, 0);
         rv = __shfl_sync(0xffffffffu, rv, 0);
         if (rk) {
             if (lane == 0) FDC_TR(ck.g, 12);
-            cursor_issue(ck, tm_k, cx.kring, cx.k_full, pol, lane);
+            cursor_issue(ck, tm_k, cx.kring, cx.k_full(), pol, lane);
             cursor_next(ck, p, cx, hi, cx.nk, lane);
         }
         if (rv) {
             if (lane == 0) FDC_TR(cv.g, 13);
-            cursor_issue(cv, tm_v, cx.vring, cx.v_full, pol, lane);
+            cursor_issue(cv, tm_v, cx.vring, cx.v_full(), pol, lane);
             cursor_next(cv, p, cx, hi, cx.nv, lane);
         }
         if (rk | rv) {
@@ -426,7 +476,7 @@ __device__ __forceinline__ void producer_loop(const AttnParams& p, const Ctx& cx
     if (!ok && lane == 0) {
         // give the copies already in flight a bounded chance to land before the CTA ends
         for (int r = 0; r < 2; ++r) {
-            const uint32_t g = r ? cv.g : ck.g, nst = r ? cx.nv : cx.nk, full = r ? cx.v_full : cx.k_full;
+            const uint32_t g = r ? cv.g : ck.g, nst = r ? cx.nv : cx.nk, full = r ? cx.v_full() : cx.k_full();
             const uint32_t first = g > nst ? g - nst : 0;
             for (uint32_t k = first; k < g; ++k) {
                 const uint32_t bar = full + 8 * (k % nst), ph = (k / nst) & 1;
@@ -458,12 +508,12 @@ __device__ __forceinline__ void qk_loop(const AttnParams& p, const Ctx& cx, long
             const int M = cx.nact[sg.s] * p.group;
             const int NP = M <= 32 ? 32 : (M <= 64 ? 64 : 128);
             const uint32_t idesc_qk = instr_desc(RROWS, NP, 0);
-            bool good = mbar_wait(cx.q_ready, seg & 1, cx.abortp, p.status);
+            bool good = mbar_wait(cx.q_ready(), seg & 1, cx.abortp, p.status);
             for (int t = 0; t < nr && good; ++t, ++g) {
-                good = mbar_wait(cx.k_full + 8 * st, kph, cx.abortp, p.status);
+                good = mbar_wait(cx.k_full() + 8 * st, kph, cx.abortp, p.status);
                 FDC_TR(g, 6);
                 const uint32_t sb = g & (cx.ns - 1);                  // score buffer of the round
-                if (good && g >= (uint32_t)cx.ns) good = mbar_wait(cx.s_free + 8 * sb, ((g / cx.ns) - 1) & 1, cx.abortp, p.status);
+                if (good && g >= (uint32_t)cx.ns) good = mbar_wait(cx.s_free() + 8 * sb, ((g / cx.ns) - 1) & 1, cx.abortp, p.status);
                 if (!good) break;
                 FDC_TR(g, 7);
                 tc_fence_after();
@@ -473,8 +523,8 @@ __device__ __forceinline__ void qk_loop(const AttnParams& p, const Ctx& cx, long
                 for (int ks = 0; ks < D / 16; ++ks)
                     umma2(d, kd + (uint32_t)(((ks >> 2) * PANEL + (ks & 3) * 32) >> 4), k_hi, q_lo + (ks >> 2) * qp16 + (uint32_t)(((ks & 3) * 32) >> 4), q_hi,
                           idesc_qk, ks > 0);
-                umma_commit(cx.k_empty + 8 * st);
-                umma_commit(cx.s_full + 8 * sb);
+                umma_commit(cx.k_empty() + 8 * st);
+                umma_commit(cx.s_full() + 8 * sb);
                 FDC_TR(g, 8);
                 if (++st == cx.nk) {
                     st = 0;
@@ -575,7 +625,7 @@ __device__ __forceinline__ void aux_loop(const AttnParams& p, const Ctx& cx, lon
                     p.stride_scene * 2, p.stride_head * 2, p.stride_row * 2, p.app_row, reinterpret_cast<const char*>(p.app_k),
                     reinterpret_cast<const char*>(p.app_v), p.tiles, p.ntile_max, p.max_active, p.hkv, p.rows, p.P, cx.pre, cx.nact, lo, hi,
                     p.status);
-        if (lane == 0) mbar_arrive(cx.app_done);
+        if (lane == 0) mbar_arrive(cx.app_done());
     }
     // The column sums of P^T (the softmax denominators), taken by the tensor core beside every
     // O^T += V^T P^T: P (128 query columns as rows, read from the same P^T buffer, which is laid out
@@ -600,8 +650,8 @@ __device__ __forceinline__ void aux_loop(const AttnParams& p, const Ctx& cx, lon
             const int ntile = sg.j1 - sg.j0;
             bool good = true;
             for (int t = 0; 2 * t < ntile && good; ++t, ++g) {
-                good = mbar_wait(cx.p_full + 8 * (g & 1), (g >> 1) & 1, cx.abortp, p.status);
-                if (good && t == 0 && seg > 0) good = mbar_wait(cx.o_free, (seg - 1) & 1, cx.abortp, p.status);
+                good = mbar_wait(cx.p_full() + 8 * (g & 1), (g >> 1) & 1, cx.abortp, p.status);
+                if (good && t == 0 && seg > 0) good = mbar_wait(cx.o_free(), (seg - 1) & 1, cx.abortp, p.status);
                 if (!good) break;
                 const uint32_t steps = (uint32_t)cx.v_steps[(g & 1) * 2] | ((uint32_t)cx.v_steps[(g & 1) * 2 + 1] << 4);
                 tc_fence_after();
@@ -613,7 +663,7 @@ __device__ __forceinline__ void aux_loop(const AttnParams& p, const Ctx& cx, lon
                         umma2(tm_l, pd + kk * 128, p_hi, ones_lo, ones_hi, idesc_sum, acc);
                         acc = 1u;
                     }
-                umma_commit(cx.pv_done + 8 * (g & 1));
+                umma_commit(cx.pv_done() + 8 * (g & 1));
             }
             ok = good;
         }
@@ -649,10 +699,10 @@ __device__ __forceinline__ void pv_loop(const AttnParams& p, const Ctx& cx, long
             const int ntile = sg.j1 - sg.j0;
             bool good = true;
             for (int t = 0; 2 * t < ntile && good; ++t, ++g) {
-                good = mbar_wait(cx.v_full + 8 * st, vph, cx.abortp, p.status);
+                good = mbar_wait(cx.v_full() + 8 * st, vph, cx.abortp, p.status);
                 FDC_TR(g, 9);
-                if (good) good = mbar_wait(cx.p_full + 8 * (g & 1), (g >> 1) & 1, cx.abortp, p.status);
-                if (good && t == 0 && seg > 0) good = mbar_wait(cx.o_free, (seg - 1) & 1, cx.abortp, p.status);
+                if (good) good = mbar_wait(cx.p_full() + 8 * (g & 1), (g >> 1) & 1, cx.abortp, p.status);
+                if (good && t == 0 && seg > 0) good = mbar_wait(cx.o_free(), (seg - 1) & 1, cx.abortp, p.status);
                 if (!good) break;
                 FDC_TR(g, 10);
                 const uint32_t steps = (uint32_t)cx.v_steps[(g & 1) * 2] | ((uint32_t)cx.v_steps[(g & 1) * 2 + 1] << 4);
@@ -673,8 +723,8 @@ __device__ __forceinline__ void pv_loop(const AttnParams& p, const Ctx& cx, long
                             acc = 1u;
                         }
                 }
-                umma_commit(cx.v_empty + 8 * st);
-                umma_commit(cx.pv_done + 8 * (g & 1));
+                umma_commit(cx.v_empty() + 8 * st);
+                umma_commit(cx.pv_done() + 8 * (g & 1));
                 FDC_TR(g, 11);
                 if (++st == cx.nv) {
                     st = 0;
@@ -880,7 +930,7 @@ __device__ __noinline__ int raise_references(const RaiseArgs a)
         if (lane < 8) wmax[q4 * 128 + a.col0 + ch * 8 + lane] = ord_of(mine);
     }
     if (tid == 0) flags[0] = 0;
-    soft_sync();
+    raise_sync(smem_u32(const_cast<int*>(a.abortp)) - RAISE_BAR_BEFORE_ABORT_FLAG, a.abortp, a.status);
     if (tid < ((np + 31) & ~31)) {                         // whole warps (the shuffles below need all lanes)
         // highest column maximum of the round (every warp of these threads computes it for itself)
         int gm = INT_MIN;
@@ -906,7 +956,7 @@ __device__ __noinline__ int raise_references(const RaiseArgs a)
             alpha[tid] = al;
         }
     }
-    soft_sync();
+    raise_sync(smem_u32(const_cast<int*>(a.abortp)) - RAISE_BAR_BEFORE_ABORT_FLAG, a.abortp, a.status);
     if (flags[0]) {                                        // a reference moved: rescale the accumulators (column sums and O^T)
         if (a.rescale_o) {
             if (!dead && !mbar_wait(a.pv_bar, a.pv_parity, a.abortp, a.status)) dead = true;   // no MMA may be writing O^T
@@ -1019,7 +1069,7 @@ __device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& 
         if (!published) {
             fence_async_smem();
             __syncwarp();
-            if (!dead && lane == 0) mbar_arrive(cx.q_ready);
+            if (!dead && lane == 0) mbar_arrive(cx.q_ready());
         }
         soft_sync();
         if (tid == 0 && seg == 0) FDC_TS(6);
@@ -1042,7 +1092,7 @@ __device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& 
             // Eq. 1 for this thread's KV row: bit i of vis <=> column col0 + i may see the row
             const uint32_t vis = masked ? row_visibility(mask_row(p, cx, seg, sg.s, 0), p.W, p.P, tile, (q4 & 1) * 32 + lane, A, G, b_lo, col0, nph) : ~0u;
             const uint32_t sb = g & (cx.ns - 1);                      // score buffer of the round
-            wait_u(cx.s_full + 8 * sb, (g / cx.ns) & 1);
+            wait_u(cx.s_full() + 8 * sb, (g / cx.ns) & 1);
             tc_fence_after();
             if (tid == 0) FDC_TR(g, 1);
             if (jb + k + 2 >= ntile && sg.next_u < hi) {
@@ -1056,8 +1106,8 @@ __device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& 
             // The P^T buffer is still being read until the PV that used it last (two rounds ago, or the
             // previous round when there is a single buffer) has completed.  Past this wait every softmax
             // warp has also finished round g - 2, so what that round left in rflag is the same for all.
-            if (cx.npb == 2) wait_u(cx.pv_done + 8 * b, ((g >> 1) & 1) ^ 1);
-            else if (g > 0) wait_u(cx.pv_done + 8 * ((g - 1) & 1), ((g - 1) >> 1) & 1);
+            if (cx.npb == 2) wait_u(cx.pv_done() + 8 * b, ((g >> 1) & 1) ^ 1);
+            else if (g > 0) wait_u(cx.pv_done() + 8 * ((g - 1) & 1), ((g - 1) >> 1) & 1);
             if (tid == 0) FDC_TR(g, 2);
             const uint32_t s_addr = cx.tmem + lane_base + sb * cx.s_stride + col0;
             // References are set in the first round of a segment.  Later a score more than 2^16 above its
@@ -1088,7 +1138,7 @@ __device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& 
                 ra.s_addr = s_addr;
                 ra.o_addr = o_addr;
                 ra.l_addr = l_addr;
-                ra.pv_bar = cx.pv_done + 8 * ((g - 1) & 1);
+                ra.pv_bar = cx.pv_done() + 8 * ((g - 1) & 1);
                 ra.pv_parity = ((g - 1) >> 1) & 1;
                 ra.vis = vis;
                 ra.c = c;
@@ -1151,7 +1201,7 @@ __device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& 
                 const int w = tile - p.P / TILE;
                 const uint64_t seen = (un && (p.P & (TILE - 1)) == 0) ? (w < p.W ? un[w] : 0ull)
                                                                        : tile_seen_rows(un, mask_row(p, cx, seg, sg.s, 0), p.W, p.P, A, tile);
-                wait_u(cx.v_full + 8 * vst, vph);
+                wait_u(cx.v_full() + 8 * vst, vph);
                 const int row = (q4 & 1) * 32 + lane;
                 const bool none = seen == 0ull;                        // (such a tile should not be listed: clear and multiply all of it)
                 const uint32_t step_seen = (uint32_t)(seen >> (row & 48)) & 0xffffu;
@@ -1178,8 +1228,8 @@ __device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& 
             fence_async_smem();
             __syncwarp();
             if (!dead && lane == 0) {
-                mbar_arrive(cx.s_free + 8 * sb);                       // the scores have been read: K Q^T may reuse the buffer
-                mbar_arrive(cx.p_full + 8 * b);
+                mbar_arrive(cx.s_free() + 8 * sb);                       // the scores have been read: K Q^T may reuse the buffer
+                mbar_arrive(cx.p_full() + 8 * b);
             }
             if (tid == 0) FDC_TR(g, 5);
         }
@@ -1203,12 +1253,12 @@ __device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& 
         }
         fence_async_smem();
         __syncwarp();
-        if (!dead && lane == 0) mbar_arrive(cx.q_ready);
+        if (!dead && lane == 0) mbar_arrive(cx.q_ready());
         prefetched = 2;
     }
     // ---- end of segment: the accumulator is final once the last PV has completed
     const uint32_t last = g - 1;
-    wait_u(cx.pv_done + 8 * (last & 1), (last >> 1) & 1);
+    wait_u(cx.pv_done() + 8 * (last & 1), (last >> 1) & 1);
     tc_fence_after();
     if (tid == 0) { FDC_TS(8); FDC_TSS(3); }
     // column sums: TMEM lane n of the accumulator of the multiplication by ones
@@ -1295,7 +1345,7 @@ __device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& 
     if (tid == 0) { FDC_TS(9); FDC_TSS(8); }
     tc_fence_before();
     __syncwarp();
-    if (!dead && lane == 0) mbar_arrive(cx.o_free);
+    if (!dead && lane == 0) mbar_arrive(cx.o_free());
 }
 
 __global__ void __launch_bounds__(THREADS, 1)
@@ -1316,19 +1366,9 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, con
     cx.qs = cx.ps + npb * cx.p_buf;
     cx.ones = cx.qs + (D / 64) * cx.q_panel;
     uint64_t* bars = reinterpret_cast<uint64_t*>(cx.ones + ONES_BYTES);
-    cx.k_full = smem_u32(bars);
-    cx.k_empty = cx.k_full + 8 * MAXST;
-    cx.v_full = cx.k_empty + 8 * MAXST;
-    cx.v_empty = cx.v_full + 8 * MAXST;
-    cx.s_full = cx.v_empty + 8 * MAXST;
-    cx.s_free = cx.s_full + 8 * 4;
-    cx.p_full = cx.s_free + 8 * 4;
+    cx.bar0 = smem_u32(bars);
     cx.ns = np_max <= 64 ? 4 : 2;
     cx.s_stride = np_max <= 64 ? 64 : 128;
-    cx.pv_done = cx.p_full + 16;
-    cx.q_ready = cx.pv_done + 16;
-    cx.o_free = cx.q_ready + 8;
-    cx.app_done = cx.o_free + 8;
     uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bars + 5 * MAXST + 16);
     cx.mneg = reinterpret_cast<float*>(tmem_holder + 4);
     cx.alpha = cx.mneg + 128;
@@ -1343,14 +1383,14 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, con
     cx.mbuf = np_max > 64 ? MBUF_MAX : MBUF;
     cx.sunion = cx.smask + 2 * cx.mbuf;
     cx.mstaged = p.max_active * p.W <= cx.mbuf;
-    __shared__ int abort_flag, v_step_bits[4];
-    cx.abortp = &abort_flag;
-    cx.v_steps = v_step_bits;
+    __shared__ CtaFlags cta_flags;
+    cx.abortp = &cta_flags.abort_flag;
+    cx.v_steps = cta_flags.v_steps;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 0) FDC_TS(0);
     if (threadIdx.x == 0) {
-        abort_flag = 0;
+        cta_flags.abort_flag = 0;
     }
     if (threadIdx.x < 4) cx.rflag[threadIdx.x] = -1;
     if (threadIdx.x < ONES_BYTES / 4 && !split_only) {
@@ -1390,22 +1430,23 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, con
     // ---- set-up that needs no global memory: barriers, TMEM
     if (threadIdx.x == 0) {
         for (int i = 0; i < MAXST; ++i) {
-            mbar_init(cx.k_full + 8 * i, 1);
-            mbar_init(cx.k_empty + 8 * i, 1);
-            mbar_init(cx.v_full + 8 * i, 1);
-            mbar_init(cx.v_empty + 8 * i, 1);
+            mbar_init(cx.k_full() + 8 * i, 1);
+            mbar_init(cx.k_empty() + 8 * i, 1);
+            mbar_init(cx.v_full() + 8 * i, 1);
+            mbar_init(cx.v_empty() + 8 * i, 1);
         }
         for (int i = 0; i < 4; ++i) {
-            mbar_init(cx.s_full + 8 * i, 1);
-            mbar_init(cx.s_free + 8 * i, NSOFT);
+            mbar_init(cx.s_full() + 8 * i, 1);
+            mbar_init(cx.s_free() + 8 * i, NSOFT);
         }
         for (int i = 0; i < 2; ++i) {
-            mbar_init(cx.p_full + 8 * i, NSOFT);
-            mbar_init(cx.pv_done + 8 * i, 2);              // the V multiplications and the column sums
+            mbar_init(cx.p_full() + 8 * i, NSOFT);
+            mbar_init(cx.pv_done() + 8 * i, 2);              // the V multiplications and the column sums
         }
-        mbar_init(cx.q_ready, NSOFT);
-        mbar_init(cx.o_free, NSOFT);
-        mbar_init(cx.app_done, 1);
+        mbar_init(cx.q_ready(), NSOFT);
+        mbar_init(cx.o_free(), NSOFT);
+        mbar_init(cx.app_done(), 1);
+        mbar_init(smem_u32(&cta_flags.raise_bar), NSOFT);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         fence_async_smem();
     }
@@ -1647,6 +1688,12 @@ attn_tc_kernel(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, con
     __syncthreads();
     if (threadIdx.x == 0) FDC_TS(10);
     if (warp == W_QK && !split_only) {
+        // TMEM is freed only when no multiplication can still be writing it.  In an orderly run they were
+        // all seen to complete before the last result was written.  After a wait that ran out, some may
+        // still be on their way: their operands are all on chip, so they finish within microseconds, and
+        // the block lingers for about a hundred before it lets go of TMEM.
+        if (*cx.abortp)
+            for (int i = 0; i < 100; ++i) __nanosleep(1000);
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(TMEM_COLS) : "memory");
     }
@@ -1688,18 +1735,9 @@ static int launch_tc(const AttnParams& p, int head_dim, cudaStream_t st, int spl
     if (rc) return rc;
     rc = get_kv_tensor_map(p.v, p, D, TILE, &tv);
     if (rc) return rc;
-    // the attribute is kept per device by the runtime
-    static size_t attr_smem[64] = {};
-    int dev = 0;
-    {
-        cudaError_t e = cudaGetDevice(&dev);
-        if (e != cudaSuccess) return set_cuda_error(e);
-    }
-    if (dev < 0 || dev >= 64 || smem > attr_smem[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return set_cuda_error(e);
-        if (dev >= 0 && dev < 64) attr_smem[dev] = smem;
-    }
+    static size_t attr_smem[kMaxDevices] = {};
+    rc = raise_dynamic_smem(reinterpret_cast<const void*>(attn_tc_kernel), smem, attr_smem);
+    if (rc) return rc;
     {
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3(p.n_cta);

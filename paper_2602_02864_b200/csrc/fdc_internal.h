@@ -137,6 +137,22 @@ int  launch_kv_append(fdc_plan* plan, const fdc_kv_desc* kv, int32_t layer, cons
                       const void* d_k_new, const void* d_v_new, void* stream);
 int  flush_pending_append(fdc_plan* plan);     // launches a recorded append on its own (no-op when there is none)
 
+// cudaFuncAttributeMaxDynamicSharedMemorySize is kept by the runtime per device: `set` remembers,
+// per device ordinal, what this process has already asked for on behalf of one kernel.
+constexpr int kMaxDevices = 64;
+inline int raise_dynamic_smem(const void* kernel, size_t bytes, size_t (&set)[kMaxDevices])
+{
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return set_cuda_error(e);
+    const bool known = dev >= 0 && dev < kMaxDevices;
+    if (known && bytes <= set[dev]) return FDC_OK;
+    e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+    if (e != cudaSuccess) return set_cuda_error(e);
+    if (known) set[dev] = bytes;
+    return FDC_OK;
+}
+
 // ----------------------------------------------------------------------------------
 // device helpers
 // ----------------------------------------------------------------------------------
