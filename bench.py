@@ -605,6 +605,14 @@ def run_fdc(args, rank: int, world: int):
         also["cfg2_fixed_rows_truncated"] = {k: (round(v, 2) if isinstance(v, float) else v) for k, v in r.items() if k in keep}
         also["cfg2_fixed_rows_truncated"]["workload"] = ("configs[2] shapes with 3-6 pre-filled field-name rows per slot (n_fixed) and no "
                                                          "lengths given: every field runs to its 96-row slot")
+        # Sec. 4.3 (future work): a fast response decoded beside the CoT.  One more source field of 24
+        # tokens: the schedule keeps its length, the first 24 passes carry one more query row per scene.
+        wd = wl.cfg2_dual_response()
+        r, _ = measure("cfg2_dual_response", args.steps, max(3, min(args.warmup, 5)), False, False, 3, w=wd)
+        also["cfg2_dual_response"] = {k: (round(v, 2) if isinstance(v, float) else v) for k, v in r.items() if k in keep}
+        also["cfg2_dual_response"]["workload"] = ("configs[2] plus one independent 24-token response field decoded concurrently "
+                                                  "(7 instead of 6 branches in the first passes)")
+        also["cfg2_dual_response"]["passes_without_the_response_field"] = main["schedule_passes"]
         also["cfg4_sweep"] = cfg4_sweep(args, device, peak)
 
     cpu = None

@@ -183,6 +183,15 @@ int fdc_build_masks(fdc_plan* plan, int32_t batch, const void* d_state, uint64_t
 int fdc_kv_append(fdc_plan* plan, const fdc_kv_desc* kv, int32_t layer, const int32_t* d_n_active,
                   const int32_t* d_kv_row, const void* d_k_new, const void* d_v_new, void* stream);
 
+/* Sec. 3.1 / Fig. 3: every line of the template starts with its field name, whose tokens are known
+ * in advance and "pre-filled".  Writes the K/V of those rows of `layer` for every scene, once, at
+ * prefill time: d_k_fixed / d_v_fixed are DEVICE [batch][hkv][F][head_dim] in the cache dtype,
+ * F = sum of n_fixed[v], rows ordered by field (template order) and then by token; row j of field v
+ * goes to cache row P + base[v] + j.  Nothing is launched for a template without fixed rows.  Rows
+ * outside [0, rows) are skipped and flagged (FDC_DEV_ROW_RANGE). */
+int fdc_kv_write_fixed(fdc_plan* plan, const fdc_kv_desc* kv, int32_t layer, const void* d_k_fixed,
+                       const void* d_v_fixed, void* stream);
+
 /* Scratch for fdc_decode_attn (split partials); depends on the plan, the cache shape and the
  * device's SM count. */
 int fdc_attn_workspace_bytes(const fdc_plan* plan, const fdc_kv_desc* kv, size_t* bytes);
@@ -200,9 +209,21 @@ int fdc_attn_workspace_bytes(const fdc_plan* plan, const fdc_kv_desc* kv, size_t
  * d_workspace: DEVICE, 256-byte aligned,
  * >= fdc_attn_workspace_bytes; its contents are undefined afterwards.
  * The tcgen05 kernel merges its split partials itself and keeps per-(scene, KV head) arrival
- * counters in the plan, and it leaves its work split there for the next call (checked against
- * d_n_active / d_ntiles before it is reused): calls that use the same plan must be ordered on
- * the GPU (one stream, or events); use one plan per concurrently decoding batch. */
+ * counters in the plan.  Its work split depends only on d_n_active / d_ntiles, so it is computed once
+ * per pass (by a small launch ahead of the pass's first attention call) and kept in the plan, checked
+ * against the counts before every use: calls that use the same plan must be ordered on the GPU (one
+ * stream, or events); use one plan per concurrently decoding batch.
+ *
+ * Reading ahead of the stream order.  The kernels are launched with programmatic stream
+ * serialization.  The first attention call on a stream after fdc_build_masks touches nothing before
+ * the kernel ahead of it has completed.  Every later attention call of the pass on that stream
+ * reads d_n_active, d_ntiles, d_tiles, d_mask, the plan's work split and the PREFIX rows (rows <
+ * prefix_len) of the cache while the kernel ahead of it may still be running; everything else (d_q,
+ * the pass's new K/V rows, cache rows >= prefix_len, the workspace, d_out) only after that kernel
+ * has completed.  Therefore: (1) the prefix rows of every layer must be complete before the pass's
+ * fdc_frontier is reached in stream order, and are never written during decoding; (2) the arrays
+ * fdc_frontier / fdc_build_masks produced must not be modified between fdc_build_masks and the last
+ * attention call of the pass. */
 int fdc_decode_attn(fdc_plan* plan, const fdc_kv_desc* kv, int32_t layer, const int32_t* d_n_active,
                     const uint64_t* d_mask, const int32_t* d_tiles, const int32_t* d_ntiles,
                     const void* d_q, void* d_out, float scale, void* d_workspace, size_t ws_bytes,
@@ -227,8 +248,10 @@ int fdc_decode_attn(fdc_plan* plan, const fdc_kv_desc* kv, int32_t layer, const 
  *     no allocating library routine); inputs and outputs are still the caller's.  Keep
  *     fdc_profile off: profiling creates CUDA events.
  *   - The FIRST call on a device looks up the buffer's device address (a host-side query made
- *     with that device current, checked, then remembered).  Make that first call during
- *     start-up, before any stream capture is begun.  The CUDA device current at the call must
+ *     with that device current, checked, then remembered); if nothing of the library has run on
+ *     that device yet, the CUDA runtime loads the library's device code at that moment, which
+ *     itself takes device memory.  Make that first call during start-up, before any stream
+ *     capture is begun; from the second call on the amount of free device memory stays put.  The CUDA device current at the call must
  *     be the plan's device (FDC_ERR_RANGE otherwise).
  *   - All calls on a GPU share the one buffer, and it keeps whatever the last call left.  No
  *     part of it has to start at zero (each call's combine pass reads only partials that the

@@ -65,6 +65,45 @@ __global__ void __launch_bounds__(128) kv_append_kernel(char* __restrict__ k, ch
     }
 }
 
+// Pre-filled field-name rows (Sec. 3.1: every line starts "field name:"; Fig. 3: those tokens are
+// "pre-filled"): fixed row i of a scene (fields in template order, then token order) goes to row
+// P + base[v] + j of the cache.  One block per (scene, fixed row); threads copy 16-byte vectors.
+__global__ void __launch_bounds__(128) kv_write_fixed_kernel(const PlanDev* __restrict__ plan, char* __restrict__ k, char* __restrict__ v,
+                                                             int64_t stride_scene_b, int64_t stride_head_b, int64_t stride_row_b, int rows,
+                                                             int hkv, int row_bytes, int n_fixed_total, const char* __restrict__ k_fixed,
+                                                             const char* __restrict__ v_fixed, int32_t* __restrict__ status)
+{
+    const int s = blockIdx.x / n_fixed_total, i = blockIdx.x - s * n_fixed_total;
+    __shared__ int s_row;
+    if (threadIdx.x == 0) {
+        int acc = 0, row = -1;
+        for (int node = 0; node < plan->n; ++node) {
+            const int nf = plan->nfixed[node];
+            if (i < acc + nf) {
+                row = plan->P + plan->base[node] + (i - acc);
+                break;
+            }
+            acc += nf;
+        }
+        if (row < 0 || row >= rows) {
+            atomicOr(status, FDC_DEV_ROW_RANGE);
+            row = -1;
+        }
+        s_row = row;
+    }
+    __syncthreads();
+    const int row = s_row;
+    if (row < 0) return;
+    const int vec_per_row = row_bytes >> 4, nvec = hkv * vec_per_row;
+    for (int x = threadIdx.x; x < nvec; x += blockDim.x) {
+        const int g = x / vec_per_row, c = x - g * vec_per_row;
+        const size_t src = (((size_t)s * hkv + g) * n_fixed_total + i) * row_bytes + (size_t)c * 16;
+        const size_t dst = (size_t)s * stride_scene_b + (size_t)g * stride_head_b + (size_t)row * stride_row_b + (size_t)c * 16;
+        *reinterpret_cast<uint4*>(k + dst) = *reinterpret_cast<const uint4*>(k_fixed + src);
+        *reinterpret_cast<uint4*>(v + dst) = *reinterpret_cast<const uint4*>(v_fixed + src);
+    }
+}
+
 }  // namespace
 
 namespace fdc {
@@ -156,4 +195,28 @@ extern "C" int fdc_kv_append(fdc_plan* p, const fdc_kv_desc* kv, int32_t layer, 
         return FDC_OK;
     }
     return launch_kv_append(p, kv, layer, d_n_active, d_kv_row, d_k_new, d_v_new, stream);
+}
+
+
+extern "C" int fdc_kv_write_fixed(fdc_plan* p, const fdc_kv_desc* kv, int32_t layer, const void* d_k_fixed, const void* d_v_fixed,
+                                  void* stream)
+{
+    int rc = check_kv_desc(p, kv, layer);
+    if (rc) return rc;
+    int total = 0;
+    for (int v = 0; v < p->h.n; ++v) total += p->h.nfixed[v];
+    if (total == 0) return FDC_OK;                 // the template has no pre-filled rows
+    if (!d_k_fixed || !d_v_fixed) return FDC_ERR_NULL;
+    if (((uintptr_t)d_k_fixed & 15) || ((uintptr_t)d_v_fixed & 15)) return FDC_ERR_SHAPE;
+    rc = flush_pending_append(p);
+    if (rc) return rc;
+    const int es = kv->dtype == FDC_F32 ? 4 : 2;
+    char* kb = (char*)kv->k + (size_t)layer * kv->stride_layer * es;
+    char* vb = (char*)kv->v + (size_t)layer * kv->stride_layer * es;
+    kv_write_fixed_kernel<<<kv->batch * total, 128, 0, (cudaStream_t)stream>>>(
+        p->d, kb, vb, (int64_t)(kv->stride_scene * es), (int64_t)(kv->stride_head * es), (int64_t)(kv->stride_row * es), (int)kv->rows,
+        (int)kv->hkv, kv->head_dim * es, total, (const char*)d_k_fixed, (const char*)d_v_fixed, p->d_status);
+    note_launch();
+    FDC_CUDA(cudaGetLastError());
+    return FDC_OK;
 }

@@ -67,6 +67,7 @@ _state_init = _sig("fdc_state_init", c_i32, c_vp, c_i32, c_vp, c_vp, c_vp)
 _frontier = _sig("fdc_frontier", c_i32, c_vp, c_i32, c_vp, c_vp, c_vp, c_vp, c_vp, c_vp, c_vp, c_vp, c_vp)
 _build_masks = _sig("fdc_build_masks", c_i32, c_vp, c_i32, c_vp, c_vp, c_vp, c_vp, c_vp, c_vp)
 _kv_append = _sig("fdc_kv_append", c_i32, c_vp, ctypes.POINTER(fdc_kv_desc), c_i32, c_vp, c_vp, c_vp, c_vp, c_vp)
+_kv_write_fixed = _sig("fdc_kv_write_fixed", c_i32, c_vp, ctypes.POINTER(fdc_kv_desc), c_i32, c_vp, c_vp, c_vp)
 _attn_ws = _sig("fdc_attn_workspace_bytes", c_i32, c_vp, ctypes.POINTER(fdc_kv_desc), ctypes.POINTER(c_sz))
 _decode_attn = _sig("fdc_decode_attn", c_i32, c_vp, ctypes.POINTER(fdc_kv_desc), c_i32, c_vp, c_vp, c_vp, c_vp,
                     c_vp, c_vp, ctypes.c_float, c_vp, c_sz, c_vp)
@@ -180,6 +181,11 @@ def fdc_build_masks(plan, batch, d_state, d_mask, d_umask, d_tiles, d_ntiles, st
 def fdc_kv_append(plan, kv: fdc_kv_desc, layer, d_n_active, d_kv_row, d_k_new, d_v_new, stream=None) -> None:
     _check(_kv_append(plan, ctypes.byref(kv), layer, _ptr(d_n_active), _ptr(d_kv_row), _ptr(d_k_new), _ptr(d_v_new),
                       _stream(stream)), "fdc_kv_append")
+
+
+def fdc_kv_write_fixed(plan, kv: fdc_kv_desc, layer, d_k_fixed, d_v_fixed, stream=None) -> None:
+    _check(_kv_write_fixed(plan, ctypes.byref(kv), layer, _ptr(d_k_fixed), _ptr(d_v_fixed), _stream(stream)),
+           "fdc_kv_write_fixed")
 
 
 def fdc_attn_workspace_bytes(plan, kv: fdc_kv_desc) -> int:
@@ -332,6 +338,10 @@ class DecodeSession:
     def kv_append(self, layer, k_new, v_new, stream=None) -> None:
         fdc_kv_append(self.plan, self.kv, layer, self.n_active, self.kv_row, k_new, v_new, self._st(stream))
         self._append_refs = (k_new, v_new)      # a recorded (fused) append reads them in the next decode_attn
+
+    def write_fixed(self, layer, k_fixed, v_fixed, stream=None) -> None:
+        """The pre-filled field-name rows of one layer: [batch][hkv][sum n_fixed][D] each."""
+        fdc_kv_write_fixed(self.plan, self.kv, layer, k_fixed, v_fixed, self._st(stream))
 
     def decode_attn(self, layer, q, out, scale, stream=None) -> None:
         fdc_decode_attn(self.plan, self.kv, layer, self.n_active, self.mask, self.tiles, self.ntiles, q, out, scale,

@@ -102,6 +102,18 @@ def cfg2_batched(layers: int = 32, batch: int = 16) -> Workload:
                     [0] * n, 6, lens, seed, 0.5)
 
 
+def cfg2_dual_response(layers: int = 32, batch: int = 16, response_len: int = 24) -> Workload:
+    """The batched configuration with one more source field, decoded beside the chain of thought
+    (Sec. 4.3, future work: a fast response produced concurrently with the comprehensive CoT).
+    The field depends on nothing and nothing depends on it: as long as it is no longer than the
+    critical path it adds width to the first passes and no pass to the schedule."""
+    w = cfg2_batched(layers, batch)
+    n = w.n_nodes
+    lens = np.concatenate([w.lens, np.full((batch, 1), response_len, np.int32)], axis=1)
+    return Workload("cfg2_dual_response_bf16", w.dtype, layers, w.hq, w.hkv, w.head_dim, batch, w.prefix_len, n + 1,
+                    list(w.edges), list(w.slot_cap) + [32], list(w.n_fixed) + [0], w.max_active + 1, lens, w.seed, w.kv_scale)
+
+
 def cfg3_wide(layers: int = 32, batch: int = 8) -> Workload:
     """Wide graph bf16: 16 leaves -> 2 aggregators (seeded 8-subsets) -> final; 48-token slots."""
     seed = BASE_SEED + 3

@@ -31,14 +31,22 @@ def alloc_cache(w: wl.Workload, device, extra_rows: int = 0, fill: float = float
     return k, v
 
 
-def write_prefix(w: wl.Workload, k, v, oracle=None, gen_device="cuda"):
+def write_prefix(w: wl.Workload, k, v, oracle=None, gen_device="cuda", sess=None):
+    """Prefill: the shared prefix rows and the pre-filled field-name rows of every layer.  With a
+    session (its cache bound) the field-name rows are placed by the library (fdc_kv_write_fixed);
+    without one they are placed here, independently."""
     for l in range(w.layers):
         pk, pv = wl.prefix_kv(w, l, gen_device)
         k[:, l, :, :w.prefix_len] = pk.to(k.device)
         v[:, l, :, :w.prefix_len] = pv.to(v.device)
         if oracle is not None:
             oracle.write_prefix(l, f32(pk), f32(pv))
-        if sum(w.n_fixed):
+        if sum(w.n_fixed) and sess is not None:
+            fk, fv = wl.fixed_kv(w, l, gen_device)
+            sess.write_fixed(l, fk.to(k.device).contiguous(), fv.to(v.device).contiguous())
+            if oracle is not None:
+                oracle.write_fixed(l, f32(fk), f32(fv))
+        elif sum(w.n_fixed):
             fk, fv = wl.fixed_kv(w, l, gen_device)
             i = 0
             base = np.concatenate([[0], np.cumsum(w.slot_cap)])
@@ -106,8 +114,8 @@ def run_and_compare(w: wl.Workload, check_steps=None, check_layers=None, extra_r
     if fused_append:          # appends are recorded and written by the attention kernel (or on their own when none follows)
         sess.set_fused_append(True)
     k, v = alloc_cache(w, device, extra_rows)
-    write_prefix(w, k, v, oracle)
     sess.bind_cache(k, v, w.hq)
+    write_prefix(w, k, v, oracle, sess=sess)
     lens_dev = torch.from_numpy(w.lens).to(device)
     sess.init(None if use_finish_flags else lens_dev)
     out = torch.zeros(w.batch, w.max_active, w.hq, w.head_dim, dtype=w.torch_dtype, device=device)

@@ -376,3 +376,56 @@ def test_more_pairs_than_thread_blocks_wide(branches):
     w = wl.cfg4_sweep(512, branches, 24)
     r = run_and_compare(w, check_steps={0, 33, 63}, fused_append=True)
     assert r["steps"] == 64 and r["checked"] > 0
+
+
+def _tail_template():
+    """A chain of thought followed by the decoding phase after it (Sec. 3.3: padding is invisible
+    "including [to] those generated for the subsequent meta-action and trajectory"; Sec. 4.1: the
+    VLA-AR head emits the trajectory as 6 tokens): four independent perception fields with long
+    slots and short contents (so that whole 64-row tiles are nothing but padding), a summary
+    that needs them all, then a meta-action field and six one-token trajectory fields, chained."""
+    n = 4 + 1 + 1 + 6
+    edges = [(i, 4) for i in range(4)] + [(4, 5)] + [(5 + i, 6 + i) for i in range(6)]
+    cap = [160, 150, 170, 160, 40, 8] + [1] * 6
+    fixed = [3, 4, 5, 6, 3, 2] + [0] * 6
+    lens = np.array([[9, 20, 12, 150, 17, 5] + [1] * 6, [30, 7, 170, 11, 40, 8] + [1] * 6], np.int32)
+    return wl.Workload("tail_phase", "bf16", 1, 8, 2, 128, 2, 200, n, edges, cap, fixed, 4, lens, 260202899, 1.0)
+
+
+def test_tail_phase_after_the_cot_sees_no_padding():
+    """The meta-action and trajectory tokens that follow the CoT see every real token of every field
+    and none of the padding; tiles that hold nothing but padding are not even visited.  Asserted on
+    the checker's tables (which the GPU tables must equal bit for bit), with attention parity on
+    those passes."""
+    from oracle import schedule as sch
+    w = _tail_template()
+    base = np.concatenate([[0], np.cumsum(w.slot_cap)])
+    tail_steps = set()
+    for s in range(w.batch):
+        lens = w.lens[s].tolist()
+        passes = sch.simulate(w.n_nodes, w.edges, lens, w.n_fixed)
+        n_tail = 0
+        for i, this in enumerate(passes):
+            if not any(v >= 5 for v, _ in this):
+                continue
+            tail_steps.add(i)
+            tab = sch.pass_tables(w.n_nodes, w.edges, w.slot_cap, lens, w.n_fixed, w.prefix_len, this)
+            for b, (v, t) in enumerate(this):
+                vis = tab["vis"][b]
+                for u in range(5 if v > 5 else v):                       # every earlier field: all of its real rows, none of its padding
+                    r0 = w.prefix_len + int(base[u])
+                    assert vis[r0:r0 + lens[u]].all() and not vis[r0 + lens[u]:r0 + w.slot_cap[u]].any()
+                n_tail += 1
+            pad_tiles = [ti for ti in range((w.rows + 63) // 64)
+                         if ti * 64 >= w.prefix_len and not tab["vis"][:, ti * 64:(ti + 1) * 64].any()]
+            assert pad_tiles and not set(pad_tiles) & set(tab["tiles"].tolist())
+        assert n_tail == (lens[5] - w.n_fixed[5]) + 6
+    r = run_and_compare(w, check_steps=tail_steps | {0, 5}, fused_append=True)
+    assert r["checked"] > 0
+
+
+def test_dual_response_template_reduced():
+    """The batched shape with a response field decoded beside the chain of thought (7 fields wide)."""
+    w = wl.cfg2_dual_response(layers=1, batch=3)
+    r = run_and_compare(w, check_steps={0, 1, 15, 16, 23, 24, 25, 60, 150}, fused_append=True)
+    assert r["checked"] > 0

@@ -280,3 +280,18 @@ def test_workload_shapes():
     assert len(sch.simulate(8, w4.edges, [64] * 8)) == 64
     w4c = wl.cfg4_sweep(1024, 8, 1, chain=True)
     assert len(sch.simulate(8, w4c.edges, [64] * 8)) == 512
+
+
+def test_a_concurrent_response_field_adds_no_pass():
+    """Sec. 4.3 (future work): a fast response decoded beside the chain of thought costs no extra
+    forward pass as long as it is shorter than the critical path: the schedule of every scene has
+    the same length with and without the extra source field, and only the first passes are wider."""
+    w0, w1 = wl.cfg2_batched(layers=1), wl.cfg2_dual_response(layers=1)
+    assert w1.n_nodes == w0.n_nodes + 1 and w1.max_active == w0.max_active + 1
+    for s in range(w0.batch):
+        p0 = sch.simulate(w0.n_nodes, w0.edges, w0.lens[s].tolist())
+        p1 = sch.simulate(w1.n_nodes, w1.edges, w1.lens[s].tolist())
+        assert len(p0) == len(p1)
+        extra = int(w1.lens[s, -1])
+        assert [len(b) - len(a) for a, b in zip(p0, p1)] == [1] * extra + [0] * (len(p0) - extra)
+        assert sch.average_parallel_degree(p1) > sch.average_parallel_degree(p0)
