@@ -37,7 +37,7 @@ NCU_TRAFFIC = {"kernel_sha256_16": "1d29deffa7da108a", "dram_bytes_per_algorithm
 
 def kernel_source_hash() -> str:
     import hashlib
-    path = os.path.join(ROOT, "paper_2602_02864_b200", "csrc", "fdc_attn_tc.cu")
+    path = os.path.join(ROOT, "paper_2602_02864_b200", "csrc", "fdc_attn_tc_kernel.cuh")
     try:
         return hashlib.sha256(open(path, "rb").read()).hexdigest()[:16]
     except OSError:
