@@ -72,11 +72,13 @@ enum {
     FDC_DEV_TIMEOUT       = 8,  /* fdc_decode_attn: a bounded in-kernel wait ran out; the    */
                                 /* launch's output is invalid                                */
     FDC_DEV_SCORE_RANGE   = 16, /* fdc_decode_attn: a score rose more than 2^100 above its   */
-                                /* softmax reference within two rounds (128 KV rows each)    */
+                                /* softmax reference within three rounds (128 KV rows each)  */
                                 /* of a reference update: the output may have overflowed     */
-    FDC_DEV_TILE_LIST     = 32  /* fdc_decode_attn: d_tiles does not list the whole prefix   */
+    FDC_DEV_TILE_LIST     = 32, /* fdc_decode_attn: d_tiles does not list the whole prefix   */
                                 /* tiles first, as entries 0, 1, 2, ... (fdc_build_masks     */
                                 /* always does); rows nobody may see could have been read    */
+    FDC_DEV_LOOP_LIMIT    = 64  /* fdc_loop_condition: max_passes reached with fields still  */
+                                /* ready: the device loop was stopped                        */
 };
 
 typedef struct fdc_plan fdc_plan;
@@ -296,6 +298,25 @@ int fdc_set_fused_append(fdc_plan* plan, int32_t on);
  * records.  At most 16384 calls are recorded between two reads. */
 int fdc_profile(fdc_plan* plan, int32_t enable);
 int fdc_profile_read(fdc_plan* plan, float* split_ms, float* combine_ms, int32_t* calls);
+
+/* Algorithm 1's loop test ("while some field is ready") for a decode loop that lives on the
+ * device: a CUDA graph whose body is a WHILE conditional node, built by the caller, with one pass
+ * of the model as the body (the caller's kernels, fdc_kv_append and fdc_decode_attn per layer,
+ * then fdc_frontier and fdc_build_masks for the NEXT pass) and this call as the body's last
+ * node.  It launches one thread that
+ *   - adds 1 to *d_pass_count (DEVICE int32 [1]; the caller zeroes it before the graph runs:
+ *     afterwards it holds the number of passes decoded),
+ *   - sets the conditional handle `cond_handle` (a cudaGraphConditionalHandle, created by the
+ *     caller for the graph the node belongs to, default value 1) to 1 if *d_all_done == 0
+ *     (fdc_frontier's output: some scene still has a ready field) and to 0 otherwise,
+ *   - and ends the loop after max_passes passes whatever d_all_done says (FDC_DEV_LOOP_LIMIT is
+ *     then set in the status word): a wrong table can never keep the GPU busy for ever.
+ * The handle is only meaningful inside a launch of its graph, so the call is for stream capture
+ * into the conditional node's body graph (or an explicit kernel node there); launched outside
+ * one it fails with a CUDA error at launch or has no effect.  Returns FDC_ERR_NULL / FDC_ERR_RANGE
+ * (max_passes < 1) / FDC_ERR_CUDA. */
+int fdc_loop_condition(fdc_plan* plan, const int32_t* d_all_done, int32_t* d_pass_count, int32_t max_passes,
+                       unsigned long long cond_handle, void* stream);
 
 /* Number of kernels this library has launched in the calling process so far. */
 int64_t fdc_launch_count(void);

@@ -186,7 +186,7 @@ __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.
 __device__ __forceinline__ void soft_sync() { asm volatile("bar.sync 1, %0;" ::"n"(NSOFT * 32) : "memory"); }
 
 // The barrier inside the reference-raising path.  Whether a warp enters that path in a given round
-// depends on data (a note left two rounds earlier), which a warp that no longer waits for anything
+// depends on data (a note left two or three rounds earlier), which a warp that no longer waits for anything
 // may read too early; a named barrier there could then be waited at for ever.  So this one is an
 // mbarrier with a bounded wait, one arrival per warp: the worst a straying warp can cause is that the
 // others give up too (FDC_DEV_TIMEOUT).
@@ -886,7 +886,7 @@ __device__ __noinline__ void merge_pair(const float* ws_ml, const float* ws_o, _
 }
 
 // The rare path of the softmax, kept out of line so that the per-round loop stays small: the
-// first round of a segment, or two rounds after some score exceeded its column's reference by
+// first round of a segment, or two (two groups: three) rounds after some score exceeded its column's reference by
 // more than 2^16.  Column maxima of the round are gathered (shuffle transpose-reduce per warp,
 // one shared-memory slot per row quadrant), references that are unset or too low are replaced,
 // alpha[n] = 2^(old - new) is published, and the column sums (TMEM) and the accumulator O^T are
@@ -1150,7 +1150,7 @@ __device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& 
             const uint32_t s_addr = cx.tmem + lane_base + sb * cx.s_stride + col0r;
             // References are set in the first round of a segment.  Later a score more than 2^16 above its
             // reference only leaves a note (no barrier in the common path): p stays far from overflow, and
-            // two rounds later, when all warps are known to see the note, the references are raised.
+            // two (two groups: three) rounds later, when all warps are known to see the note, the references are raised.
             if (t == 0 && __shfl_sync(0xffffffffu, my_tile, k & 31) * TILE + TILE <= p.P) {
                 // First round of a segment inside the prefix: every column takes its score against the
                 // round's first KV row (visible to all) as reference.  That row's own term is then exactly

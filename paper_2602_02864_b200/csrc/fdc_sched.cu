@@ -226,6 +226,21 @@ __global__ void __launch_bounds__(256) build_masks_kernel(const PlanDev* __restr
     (void)T;
 }
 
+// Algorithm 1's loop test, on the device: keeps a WHILE node of a CUDA graph going while some scene
+// still has a ready field.
+__global__ void loop_condition_kernel(const int32_t* __restrict__ all_done, int32_t* __restrict__ pass_count,
+                                      int32_t max_passes, cudaGraphConditionalHandle handle, int32_t* __restrict__ status)
+{
+    const int32_t done_passes = *pass_count + 1;      // the pass whose tables were just replaced has been decoded
+    *pass_count = done_passes;
+    unsigned int more = *all_done == 0 ? 1u : 0u;
+    if (more && done_passes >= max_passes) {           // never an endless loop, whatever the tables say
+        more = 0u;
+        atomicOr(status, FDC_DEV_LOOP_LIMIT);
+    }
+    cudaGraphSetConditional(handle, more);
+}
+
 }  // namespace
 
 extern "C" {
@@ -280,6 +295,22 @@ int fdc_build_masks(fdc_plan* p, int32_t batch, const void* d_state, uint64_t* d
     ++p->tables_gen;                       // the pass tables change: work splits made from them are stale
     build_masks_kernel<<<batch, 256, p->h.W * sizeof(uint64_t), (cudaStream_t)stream>>>(
         p->d, (const SceneState*)d_state, d_mask, d_umask, d_tiles, d_ntiles);
+    note_launch();
+    FDC_CUDA(cudaGetLastError());
+    return FDC_OK;
+}
+
+int fdc_loop_condition(fdc_plan* p, const int32_t* d_all_done, int32_t* d_pass_count, int32_t max_passes,
+                       unsigned long long cond_handle, void* stream)
+{
+    if (!p || !d_all_done || !d_pass_count) return FDC_ERR_NULL;
+    if (max_passes < 1) return FDC_ERR_RANGE;
+    {
+        int rcf = flush_pending_append(p);
+        if (rcf) return rcf;
+    }
+    loop_condition_kernel<<<1, 1, 0, (cudaStream_t)stream>>>(d_all_done, d_pass_count, max_passes,
+                                                             (cudaGraphConditionalHandle)cond_handle, p->d_status);
     note_launch();
     FDC_CUDA(cudaGetLastError());
     return FDC_OK;

@@ -30,6 +30,7 @@ FDC_F32, FDC_BF16 = 0, 1
 FDC_DEV_ROW_RANGE, FDC_DEV_FRONTIER_WIDE, FDC_DEV_LEN_RANGE, FDC_DEV_TIMEOUT = 1, 2, 4, 8
 FDC_DEV_SCORE_RANGE = 16
 FDC_DEV_TILE_LIST = 32
+FDC_DEV_LOOP_LIMIT = 64
 
 c_i32, c_i64, c_vp, c_sz = ctypes.c_int32, ctypes.c_int64, ctypes.c_void_p, ctypes.c_size_t
 
@@ -78,6 +79,7 @@ _set_attn_kernel = _sig("fdc_set_attn_kernel", c_i32, c_vp, c_i32)
 _set_fused_append = _sig("fdc_set_fused_append", c_i32, c_vp, c_i32)
 _kernel_name = _sig("fdc_kernel_name", ctypes.c_char_p, c_i32)
 _profile = _sig("fdc_profile", c_i32, c_vp, c_i32)
+_loop_condition = _sig("fdc_loop_condition", c_i32, c_vp, c_vp, c_vp, c_i32, ctypes.c_uint64, c_vp)
 _profile_read = _sig("fdc_profile_read", c_i32, c_vp, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_float),
                      ctypes.POINTER(c_i32))
 _launch_count = _sig("fdc_launch_count", c_i64)
@@ -226,6 +228,11 @@ def fdc_set_attn_kernel(plan, which: int) -> None:
 
 def fdc_set_fused_append(plan, on: bool) -> None:
     _check(_set_fused_append(plan, 1 if on else 0), "fdc_set_fused_append")
+
+
+def fdc_loop_condition(plan, d_all_done, d_pass_count, max_passes: int, cond_handle: int, stream=None) -> None:
+    _check(_loop_condition(plan, _ptr(d_all_done), _ptr(d_pass_count), int(max_passes), int(cond_handle), _stream(stream)),
+           "fdc_loop_condition")
 
 
 def fdc_kernel_name(which: int) -> Optional[str]:
