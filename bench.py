@@ -387,6 +387,10 @@ def run_fdc(args, rank: int, world: int):
     torch.cuda.set_device(local)
     device = torch.device("cuda", local)
     peak, peak_src = measured_peaks()
+    if args.only_device_loop:
+        if rank == 0:
+            print(json.dumps({"device_loop": device_loop_report(args.workload, device)}), flush=True)
+        return
 
     def measure(name: str, K: int, W: int, with_e2e: bool, sample_clocks: bool, reps: int, w=None):
         w = get_workload(name) if w is None else w
@@ -614,6 +618,7 @@ def run_fdc(args, rank: int, world: int):
                                                   "(7 instead of 6 branches in the first passes)")
         also["cfg2_dual_response"]["passes_without_the_response_field"] = main["schedule_passes"]
         also["cfg4_sweep"] = cfg4_sweep(args, device, peak)
+        also["device_loop"] = device_loop_report(args.workload, device)
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu:
@@ -646,6 +651,68 @@ def run_fdc(args, rank: int, world: int):
             "paper_context": "paper reports 3.1-4.1x CoT speedup end to end on 1x A100 80GB (bf16); no kernel-level number",
         }
         print(json.dumps(line), flush=True)
+
+
+def device_loop_report(name: str, device):
+    """Algorithm 1's whole loop as ONE graph launch (a WHILE node kept going by fdc_loop_condition)
+    against the same passes replayed from the host as one graph each.  Both decode the workload's
+    whole schedule from fdc_state_init to the last pass with one set of per-pass inputs; timed with
+    CUDA events from the reset to the end, median of 3."""
+    import torch
+    from paper_2602_02864_b200.device_loop import DeviceLoop
+    w = get_workload(name)
+    n_pass = schedule_length(w)
+    sb = StepBench(w, 1, device)
+    stream = torch.cuda.current_stream()
+    sb.sess.use_stream(stream)
+    sb.reset()
+    sb.step(0)                                   # eager once
+    torch.cuda.synchronize()
+    sb.sess.use_stream(None)
+    g = sb.capture(0)                            # frontier + build_masks + layers x (append, attention)
+
+    def body(st):
+        sb.layers_pass(0)
+        sb.schedule_pass()
+
+    loop = DeviceLoop(sb.sess, body, int(sum(w.slot_cap)))
+    sb.sess.use_stream(stream)
+
+    def run_host():
+        sb.reset()
+        for _ in range(n_pass):
+            g.replay()
+
+    def run_device():
+        sb.reset()
+        sb.schedule_pass()
+        loop.launch(stream)
+
+    res = {}
+    for key, fn in (("host_replays_one_graph_per_pass", run_host), ("device_loop_one_graph_launch", run_device)):
+        fn()
+        torch.cuda.synchronize()
+        ts = []
+        for _ in range(3):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            fn()
+            e1.record(stream)
+            torch.cuda.synchronize()
+            ts.append(e0.elapsed_time(e1))
+        ms = sorted(ts)[1]
+        res[key] = {"whole_schedule_ms": round(ms, 3), "layer_step_us": round(ms / n_pass / w.layers * 1e3, 2)}
+    res["passes_by_host_arithmetic"] = n_pass
+    res["passes_counted_on_device"] = int(loop.passes.item())
+    res["device_status"] = sb.sess.status(clear=True)
+    res["workload"] = WORKLOAD_TEXT[name] + "; every pass reads the same q / k_new / v_new buffers"
+    sb.sess.use_stream(None)
+    loop.close()
+    sb.graphs.clear()
+    sb.sess.close()
+    del sb
+    torch.cuda.empty_cache()
+    return res
 
 
 # configs[4]: prefix x branches x scenes.  A bounded part of the grid: every prefix x branches at 8
@@ -806,6 +873,7 @@ def main():
     ap.add_argument("--workload", default="cfg2", choices=["cfg0", "cfg1", "cfg2", "cfg3"])
     ap.add_argument("--impl", default="fdc", choices=["fdc", "reference"])
     ap.add_argument("--no-also", action="store_true", help="skip the short runs of the other configurations")
+    ap.add_argument("--only-device-loop", action="store_true", help="run only the whole-schedule comparison (host-replayed graphs vs one device loop)")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU baseline leg")
     ap.add_argument("--separate-append", action="store_true",
                     help="launch kv_append as a kernel of its own instead of inside the attention kernel")
