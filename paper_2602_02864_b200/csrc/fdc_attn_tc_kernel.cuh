@@ -1464,7 +1464,7 @@ FDC_TC_KERNEL(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, cons
     // was computed from.  The memo's loads and those of the counts are all issued before the first
     // use, so that they share one trip to memory; when they may be read ahead of the dependency wait
     // they are issued right here, and the trip hides behind the set-up.
-    constexpr int MEMO_MAGIC = 0x5D170000 | (W_PREFIX << 12) | (W_MASKED << 8) | W_PAIR;
+    constexpr int MEMO_MAGIC = 0x5D180000 | (W_PREFIX << 12) | (W_MASKED << 8) | W_PAIR;
     const int32_t* mrd = (p.split_memo && !split_only) ? p.split_memo : nullptr;
     int4 mh0 = make_int4(0, 0, 0, 0), mh1 = mh0, mh2 = mh0, me = mh0;
     int m_na = -1, m_nt = -1, m_prev = 0;
@@ -1629,6 +1629,21 @@ FDC_TC_KERNEL(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, cons
             }
         } else if (threadIdx.x == 0) {
             split_tpart = 0;
+        }
+        __syncthreads();
+        if (one_part && threadIdx.x == 0) {
+            // One part per CTA leaves CTAs idle when the parts per pair do not divide the CTAs evenly
+            // (64 pairs on 148 CTAs: 2 or 3 parts, a CTA carries up to 16 % more than the average).  Where the
+            // shares are long enough for a pair boundary inside a CTA to cost less than that (measured:
+            // from about 200 prefix tiles per CTA, half of that with 128 query rows, whose rounds take twice
+            // as long), equal shares of the weighted length win after all.
+            long long tot = 0;
+            for (int i = 0; i < p.batch; ++i) {
+                const int nt = cx.pre[i + 1] - cx.pre[i];
+                if (nt > 0) tot += vt_of(cx, nt, nt) + W_PAIR;
+            }
+            const long long avg = tot * p.hkv / p.n_cta;
+            if (avg * (np_max > 64 ? 2 : 1) >= 200 * W_PREFIX && (long long)split_tpart * 100 > avg * 108) split_tpart = 0;
         }
         __syncthreads();
         if (threadIdx.x < 32) {
