@@ -1,7 +1,8 @@
 """Exact-integer checker: field DAG, Algorithm 1 schedule, slots, visibility, bitmaps.
 
 TEST INFRASTRUCTURE ONLY (see the package docstring).  Notation follows the paper:
-G = (V, E), d_v = remaining unfinished prerequisites of v, S = ready set.
+G = (V, E); the ready set S of Algorithm 1 is, in every pass, the set of unfinished fields whose
+prerequisites have all finished.
 
 Readings taken where the paper is silent (Sec. 3.2 - 3.3 leave these open):
   * a newly ready field first decodes in the NEXT forward pass (Alg. 1: decoding is the
@@ -87,34 +88,28 @@ def slot_base(slot_cap: Sequence[int]) -> List[int]:
 
 def simulate(n: int, edges: Sequence[Tuple[int, int]], lens: Sequence[int],
              n_fixed: Sequence[int] | None = None) -> List[List[Tuple[int, int]]]:
-    """Algorithm 1, taken literally.  Returns, per forward pass, the packed list of
-    (v, t): field v decodes its token t in that pass (ascending v)."""
+    """The schedule Algorithm 1 (Sec. 3.2) produces, written as its defining property instead of
+    the listing's bookkeeping: in every forward pass exactly those fields decode one token that
+    are unfinished and whose prerequisites had all finished BEFORE the pass; a field is finished
+    once it holds lens[v] rows.  Returns, per forward pass, the packed list of (v, t): field v
+    decodes its token t in that pass (ascending v)."""
     validate(n, edges)
     n_fixed = [0] * n if n_fixed is None else list(n_fixed)
     for v in range(n):
         if not (n_fixed[v] + 1 <= lens[v]):
             raise GraphError("every field must generate at least one token")
-    d = [0] * n                                   # d_v <- number of incoming edges
-    for (_, b) in edges:
-        d[b] += 1
-    S = {v for v in range(n) if d[v] == 0}        # ready set <- sources
-    tok = [n_fixed[v] for v in range(n)]          # rows of v already in the cache
+    parents: List[List[int]] = [[a for (a, b) in edges if b == v] for v in range(n)]
+    rows = [n_fixed[v] for v in range(n)]         # rows of v already in the cache
     passes: List[List[Tuple[int, int]]] = []
-    while S:
-        this_pass = []
-        for v in sorted(S):                       # one new token in every ready field
-            this_pass.append((v, tok[v]))
-            tok[v] += 1
-        passes.append(this_pass)
-        for v in sorted(S):
-            if tok[v] == lens[v]:                 # field finished
-                S.remove(v)                       # leaves the ready set
-                for (a, u) in edges:              # every edge (v, u)
-                    if a == v:
-                        d[u] -= 1
-                        if d[u] == 0:
-                            S.add(u)              # decodes from the next pass on
-    if any(tok[v] != lens[v] for v in range(n)):
+    while True:
+        finished = [rows[v] == lens[v] for v in range(n)]          # state before this pass
+        ready = [v for v in range(n) if not finished[v] and all(finished[u] for u in parents[v])]
+        if not ready:
+            break
+        passes.append([(v, rows[v]) for v in ready])
+        for v in ready:
+            rows[v] += 1
+    if any(rows[v] != lens[v] for v in range(n)):
         raise GraphError("schedule did not complete")
     return passes
 
