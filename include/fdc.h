@@ -318,6 +318,15 @@ int fdc_profile_read(fdc_plan* plan, float* split_ms, float* combine_ms, int32_t
 int fdc_loop_condition(fdc_plan* plan, const int32_t* d_all_done, int32_t* d_pass_count, int32_t max_passes,
                        unsigned long long cond_handle, void* stream);
 
+/* Self-test of the bounded wait that every in-kernel wait of the attention kernels goes through
+ * (an mbarrier poll with an iteration limit; when the limit is reached the thread raises its
+ * block's abort flag, sets FDC_DEV_TIMEOUT and goes on without waiting).  Launches one block of
+ * 64 threads that wait for a barrier nothing will ever complete; the launch ends by itself (about
+ * a second), *d_outcome (DEVICE int32 [1]) receives the number of threads whose wait gave up (64)
+ * and the plan's status word gets FDC_DEV_TIMEOUT, to be read and cleared with fdc_status.
+ * For start-up checks and tests; nothing else in the library calls it. */
+int fdc_selftest_bounded_wait(fdc_plan* plan, int32_t* d_outcome, void* stream);
+
 /* Number of kernels this library has launched in the calling process so far. */
 int64_t fdc_launch_count(void);
 

@@ -8,7 +8,7 @@
 
 namespace fdc {
 
-constexpr uint32_t SPIN_LIMIT = 1u << 22;
+constexpr uint32_t SPIN_LIMIT = 1u << 18;      // polls of a bounded wait: about a second (a poll that finds the phase incomplete is suspended for a few microseconds by the hardware)
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 

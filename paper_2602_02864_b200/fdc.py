@@ -79,6 +79,7 @@ _set_attn_kernel = _sig("fdc_set_attn_kernel", c_i32, c_vp, c_i32)
 _set_fused_append = _sig("fdc_set_fused_append", c_i32, c_vp, c_i32)
 _kernel_name = _sig("fdc_kernel_name", ctypes.c_char_p, c_i32)
 _profile = _sig("fdc_profile", c_i32, c_vp, c_i32)
+_selftest_bounded_wait = _sig("fdc_selftest_bounded_wait", c_i32, c_vp, c_vp, c_vp)
 _loop_condition = _sig("fdc_loop_condition", c_i32, c_vp, c_vp, c_vp, c_i32, ctypes.c_uint64, c_vp)
 _profile_read = _sig("fdc_profile_read", c_i32, c_vp, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_float),
                      ctypes.POINTER(c_i32))
@@ -228,6 +229,10 @@ def fdc_set_attn_kernel(plan, which: int) -> None:
 
 def fdc_set_fused_append(plan, on: bool) -> None:
     _check(_set_fused_append(plan, 1 if on else 0), "fdc_set_fused_append")
+
+
+def fdc_selftest_bounded_wait(plan, d_outcome, stream=None) -> None:
+    _check(_selftest_bounded_wait(plan, _ptr(d_outcome), _stream(stream)), "fdc_selftest_bounded_wait")
 
 
 def fdc_loop_condition(plan, d_all_done, d_pass_count, max_passes: int, cond_handle: int, stream=None) -> None:

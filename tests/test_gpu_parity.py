@@ -437,3 +437,23 @@ def test_dual_response_template_reduced():
     w = wl.cfg2_dual_response(layers=1, batch=3)
     r = run_and_compare(w, check_steps={0, 1, 15, 16, 23, 24, 25, 60, 150}, fused_append=True)
     assert r["checked"] > 0
+
+
+def test_a_wait_that_cannot_end_gives_up_and_is_reported():
+    """The bounded wait of the attention kernels, run against a barrier that nothing completes
+    (fdc_selftest_bounded_wait): the launch ends by itself, every waiting thread gave up, the
+    status word says FDC_DEV_TIMEOUT, and after clearing it the next ordinary run is correct."""
+    from paper_2602_02864_b200 import fdc
+    w = wl.cfg0_tiny()
+    sess = fdc.DecodeSession(w.n_nodes, w.edges, w.slot_cap, w.n_fixed, w.prefix_len, w.max_active, w.batch, "cuda")
+    outcome = torch.zeros(1, dtype=torch.int32, device="cuda")
+    fdc.fdc_selftest_bounded_wait(sess.plan, outcome)
+    torch.cuda.synchronize()
+    assert int(outcome.item()) == 64
+    assert sess.status(clear=True) == fdc.FDC_DEV_TIMEOUT
+    assert sess.status() == 0
+    sess.close()
+    w2 = wl.cfg0_tiny()
+    w2.dtype, w2.head_dim = "bf16", 128
+    r = run_and_compare(w2, check_steps={0, 1, 5})
+    assert r["checked"] > 0
