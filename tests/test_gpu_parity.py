@@ -457,3 +457,24 @@ def test_a_wait_that_cannot_end_gives_up_and_is_reported():
     w2.dtype, w2.head_dim = "bf16", 128
     r = run_and_compare(w2, check_steps={0, 1, 5})
     assert r["checked"] > 0
+
+
+@pytest.mark.parametrize("case", range(16))
+def test_random_templates_larger_shapes(case):
+    """Random DAGs on shapes the small random cases do not reach: GQA groups of 1 to 16, up to 24
+    parallel fields (all three query-row widths of the tcgen05 kernel), 1 to 40 scenes (fewer and
+    more (scene, KV head) pairs than thread blocks), prefixes of 0 to 3000 rows, slots of up to 130
+    rows; the first, some middle and the last passes are compared."""
+    from oracle import schedule as sch
+    rng = np.random.default_rng(77000 + case)
+    G = int(rng.choice([1, 2, 4, 7, 8, 16]))
+    hkv = int(rng.choice([1, 2, 4, 8]))
+    n_nodes = int(rng.integers(2, min(24, 128 // G) + 1))
+    batch = int(rng.choice([1, 2, 5, 19, 24, 40]))
+    w = wl.random_template(int(rng.integers(1 << 30)), n_nodes=n_nodes, edge_prob=float(rng.choice([0.0, 0.15, 0.4])), cap_lo=2,
+                           cap_hi=int(rng.choice([6, 40, 70, 130])), batch=batch, prefix_len=int(rng.choice([0, 64, 100, 640, 1000, 2048, 3000])),
+                           fixed_hi=int(rng.integers(0, 3)), hq=hkv * G, hkv=hkv, head_dim=128, dtype="bf16")
+    w.max_active = n_nodes
+    n = max(len(sch.simulate(w.n_nodes, w.edges, w.lens[s].tolist(), w.n_fixed)) for s in range(w.batch))
+    r = run_and_compare(w, check_steps={0, 1, 2, n // 3, n // 2, n - 2, n - 1}, fused_append=bool(rng.integers(2)), kernel=3)
+    assert r["steps"] == n and r["checked"] > 0
