@@ -36,8 +36,8 @@
 // later (no barrier in the common path); a rise of more than 2^100 within those rounds is
 // flagged.  Sums and accumulator use the same reference and the same rounded P^T, so the result
 // is exact up to the rounding of P^T.
-#ifndef FDC_TC_NGRP
-#error "include from a translation unit that defines FDC_TC_NGRP (1 or 2), FDC_TC_KERNEL and FDC_TC_LAUNCH"
+#if !defined(FDC_TC_NGRP) || !defined(FDC_TC_NPMAX)
+#error "include from a translation unit that defines FDC_TC_NGRP (1 or 2), FDC_TC_NPMAX (32, 64 or 128), FDC_TC_KERNEL and FDC_TC_LAUNCH"
 #endif
 #include <cudaTypedefs.h>
 
@@ -53,6 +53,8 @@ constexpr int D = 128;                       // head_dim handled by this kernel
 constexpr int TILE = FDC_TILE_ROWS;          // rows per entry of the visited-tile list
 constexpr int RROWS = 2 * TILE;              // KV rows per round = M of S^T = K of O^T
 constexpr int NGRP = FDC_TC_NGRP;            // groups the softmax warps work in (this build)
+constexpr int NP_MAX = FDC_TC_NPMAX;         // padded query rows of the widest pair of the launches this build serves (32, 64 or 128)
+static_assert((NP_MAX == 64) == (NGRP == 2), "two groups exactly for 33 to 64 query rows");
 constexpr int NSOFT = 16;                    // softmax warps: 4 row quadrants x 4 column parts
 constexpr int NPART = NSOFT / 4;             // column parts
 constexpr int W_PROD = NSOFT, W_QK = NSOFT + 1, W_AUX = NSOFT + 2, W_PV = NSOFT + 3;
@@ -516,7 +518,7 @@ __device__ __forceinline__ void qk_loop(const AttnParams& p, const Ctx& cx, long
         const int nr = (sg.j1 - sg.j0 + 1) >> 1;
         if (lane == 0) {
             const int M = cx.nact[sg.s] * p.group;
-            const int NP = M <= 32 ? 32 : (M <= 64 ? 64 : 128);
+            const int NP = (NP_MAX == 32 || M <= 32) ? 32 : ((NP_MAX == 64 || M <= 64) ? 64 : 128);
             const uint32_t idesc_qk = instr_desc(RROWS, NP, 0);
             bool good = mbar_wait(cx.q_ready(), seg & 1, cx.abortp, p.status);
             for (int t = 0; t < nr && good; ++t, ++g) {
@@ -704,7 +706,7 @@ __device__ __forceinline__ void pv_loop(const AttnParams& p, const Ctx& cx, long
         const Segment sg = decode_segment(u, hi, cx.pre, p.hkv, s);
         if (lane == 0) {
             const int M = cx.nact[sg.s] * p.group;
-            const int NP = M <= 32 ? 32 : (M <= 64 ? 64 : 128);
+            const int NP = (NP_MAX == 32 || M <= 32) ? 32 : ((NP_MAX == 64 || M <= 64) ? 64 : 128);
             const uint32_t idesc_pv = instr_desc(D, NP, 1);
             const int ntile = sg.j1 - sg.j0;
             bool good = true;
@@ -785,7 +787,7 @@ __device__ __noinline__ void prefetch_next_segment(const uint4* qg, const uint64
     int s2 = s_cur;
     const Segment nx = decode_segment(next_u, hi, pre, hkv, s2);
     const int M2 = nact[nx.s] * G;
-    const int NP2 = M2 <= 32 ? 32 : (M2 <= 64 ? 64 : 128);
+    const int NP2 = (NP_MAX == 32 || M2 <= 32) ? 32 : ((NP_MAX == 64 || M2 <= 64) ? 64 : 128);
     for (int idx = tid; idx < NP2 * (D / 8); idx += NSOFT * 32) {
         const int n = idx / (D / 8), ch = idx - n * (D / 8);
         const bool valid = n < M2;
@@ -807,7 +809,7 @@ __device__ __noinline__ void stage_first_pair_early(const uint4* qg, const uint6
                                                     unsigned char* qs, int q_panel, uint64_t* smask_dst)
 {
     const int tid = threadIdx.x;
-    const int NP = M <= 32 ? 32 : (M <= 64 ? 64 : 128);
+    const int NP = (NP_MAX == 32 || M <= 32) ? 32 : ((NP_MAX == 64 || M <= 64) ? 64 : 128);
     if (smask_dst) {
         const uint64_t* src = mask + (size_t)s * max_active * W;
         for (int idx = tid; idx < max_active * W; idx += NSOFT * 32) smask_dst[idx] = src[idx];
@@ -1412,13 +1414,14 @@ __device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& 
 
 __global__ void __launch_bounds__(THREADS, 1)
 FDC_TC_KERNEL(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
-               const int nk, const int nv, const int np_max, const int npb, const int split_only)
+               const int nk, const int nv, const int split_only)
 {
     extern __shared__ unsigned char smem_dyn[];
     unsigned char* smem = reinterpret_cast<unsigned char*>(((uintptr_t)smem_dyn + 1023) & ~(uintptr_t)1023);
     Ctx cx;
     cx.nk = nk;
     cx.nv = nv;
+    constexpr int np_max = NP_MAX, npb = NP_MAX > 64 ? 1 : 2;      // (128 query rows: one P^T buffer, so that four stages still fit)
     cx.q_panel = np_max * 128;
     cx.p_buf = ((np_max + 63) / 64) * PANEL;
     cx.npb = npb;
@@ -1755,7 +1758,7 @@ FDC_TC_KERNEL(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, cons
         while (u < hi) {
             const Segment sg = decode_segment(u, hi, cx.pre, p.hkv, s);
             const int M = cx.nact[sg.s] * p.group;
-            softmax_segment(p, cx, sg, (M <= 32 ? 32 : (M <= 64 ? 64 : 128)) / NPART, seg, hi, prefetched, g, vst, vph, dead, warp, lane);
+            softmax_segment(p, cx, sg, ((NP_MAX == 32 || M <= 32) ? 32 : ((NP_MAX == 64 || M <= 64) ? 64 : 128)) / NPART, seg, hi, prefetched, g, vst, vph, dead, warp, lane);
             ++seg;
             u = sg.next_u;
         }
@@ -1799,6 +1802,7 @@ int FDC_TC_LAUNCH(const AttnParams& p, int head_dim, cudaStream_t st, int split_
     if (head_dim != D || p.mmax > 128) return FDC_ERR_SHAPE;
     const int np_max = p.mmax <= 32 ? 32 : (p.mmax <= 64 ? 64 : 128);
     const int p_buf = ((np_max + 63) / 64) * PANEL;
+    if (np_max != NP_MAX) return FDC_ERR_SHAPE;   // another build's launches
     const int npb = np_max > 64 ? 1 : 2;          // 128 query rows: one P^T buffer, so that four stages still fit
     const size_t fixed = 1024 + (size_t)npb * p_buf + (size_t)(D / 64) * np_max * 128 + ONES_BYTES + 8 * (5 * MAXST + 16) + 16 +
                          4 * (128 + 128 + 512 + 128 + 12) + sizeof(int) * (3 * p.batch + 2) + 8 * (2 * (np_max > 64 ? MBUF_MAX : MBUF) + 2 * UW + 2) + 64;
@@ -1813,7 +1817,6 @@ int FDC_TC_LAUNCH(const AttnParams& p, int head_dim, cudaStream_t st, int split_
     if (rc) return rc;
     rc = get_kv_tensor_map(p.v, p, D, TILE, &tv);
     if (rc) return rc;
-    if ((np_max == 64) != (NGRP == 2)) return FDC_ERR_SHAPE;      // the other build's launches
     static size_t attr_smem[kMaxDevices] = {};
     rc = raise_dynamic_smem(reinterpret_cast<const void*>(FDC_TC_KERNEL), smem, attr_smem);
     if (rc) return rc;
@@ -1828,7 +1831,7 @@ int FDC_TC_LAUNCH(const AttnParams& p, int head_dim, cudaStream_t st, int split_
         at[0].val.programmaticStreamSerializationAllowed = 1;
         cfg.attrs = at;
         cfg.numAttrs = split_only ? 0 : 1;
-        cudaError_t e = cudaLaunchKernelEx(&cfg, FDC_TC_KERNEL, p, tk, tv, nk, nv, np_max, npb, split_only);
+        cudaError_t e = cudaLaunchKernelEx(&cfg, FDC_TC_KERNEL, p, tk, tv, nk, nv, split_only);
         if (e != cudaSuccess) return set_cuda_error(e);
     }
     note_launch();
