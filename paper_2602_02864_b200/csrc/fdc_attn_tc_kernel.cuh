@@ -1424,6 +1424,9 @@ FDC_TC_KERNEL(const AttnParams p, const __grid_constant__ CUtensorMap tm_k, cons
     constexpr int np_max = NP_MAX, npb = NP_MAX > 64 ? 1 : 2;      // (128 query rows: one P^T buffer, so that four stages still fit)
     cx.q_panel = np_max * 128;
     cx.p_buf = ((np_max + 63) / 64) * PANEL;
+    // (register allocation: with this one value folded into the address arithmetic the two wider builds
+    // spill; kept in a register they do not, or hardly)
+    if (NP_MAX > 32) asm volatile("" : "+r"(cx.p_buf));
     cx.npb = npb;
     cx.kring = smem;
     cx.vring = cx.kring + (size_t)nk * STAGE;
