@@ -1052,7 +1052,7 @@ __device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& 
         } else {
             // all global reads first (one latency), then the stores
             const uint4* qg = reinterpret_cast<const uint4*>(p.q);
-            constexpr int QPT = 128 * (D / 8) / (NSOFT * 32);      // 16-byte chunks per thread for 128 query rows
+            constexpr int QPT = NP_MAX * (D / 8) / (NSOFT * 32);   // 16-byte chunks per thread for the widest pair of this build
             uint4 qv[QPT];
 #pragma unroll
             for (int i = 0; i < QPT; ++i) {
@@ -1064,10 +1064,10 @@ __device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& 
                     qv[i] = qg[((((size_t)sg.s * p.max_active + b) * p.hq + (size_t)sg.g * G + hg) * D) / 8 + ch];
                 }
             }
-            uint64_t mv[MBUF_MAX / (NSOFT * 32)];
+            uint64_t mv[(NP_MAX > 64 ? MBUF_MAX : MBUF) / (NSOFT * 32)];
             const int nw = cx.mstaged ? p.max_active * p.W : 0;
 #pragma unroll
-            for (int i = 0; i < MBUF_MAX / (NSOFT * 32); ++i) {
+            for (int i = 0; i < (NP_MAX > 64 ? MBUF_MAX : MBUF) / (NSOFT * 32); ++i) {
                 const int idx = tid + i * (NSOFT * 32);
                 mv[i] = idx < nw ? p.mask[(size_t)sg.s * p.max_active * p.W + idx] : 0ull;
             }
@@ -1078,7 +1078,7 @@ __device__ __forceinline__ void softmax_segment(const AttnParams& p, const Ctx& 
                 if (n < np) *reinterpret_cast<uint4*>(cx.qs + (ch >> 3) * cx.q_panel + n * 128 + (((ch & 7) ^ (n & 7)) << 4)) = qv[i];
             }
 #pragma unroll
-            for (int i = 0; i < MBUF_MAX / (NSOFT * 32); ++i) {
+            for (int i = 0; i < (NP_MAX > 64 ? MBUF_MAX : MBUF) / (NSOFT * 32); ++i) {
                 const int idx = tid + i * (NSOFT * 32);
                 if (idx < nw) cx.smask[(seg & 1) * cx.mbuf + idx] = mv[i];
             }
