@@ -32,7 +32,7 @@ sys.path.insert(0, ROOT)
 # profiles/attn_tc_kernel_cfg2.md (dram__bytes_read.sum + dram__bytes_write.sum over the launch's
 # algorithmic bytes; traffic grows in proportion to the visited tiles, so it scales to a full-size
 # launch).  Only valid for the kernel source it was measured on: keyed by a hash of that source.
-NCU_TRAFFIC = {"kernel_sha256_16": "6e6429e607018b0c", "dram_bytes_per_algorithmic_byte": 1.095}
+NCU_TRAFFIC = {"kernel_sha256_16": "131986594b3087ed", "dram_bytes_per_algorithmic_byte": 1.096}
 
 
 def kernel_source_hash() -> str:
